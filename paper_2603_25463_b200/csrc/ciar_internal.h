@@ -1,0 +1,62 @@
+// Internal interface between the host entry points (api.cu) and the kernel launchers.
+#pragma once
+
+#include "ciar_device.cuh"
+
+namespace ciar {
+
+struct QuantifyArgs {
+    const void *logits;
+    int64_t rows;  // logical rows of this launch
+    int64_t row_stride;
+    int32_t vb, n;
+    RowMap rm;
+    int32_t radius_mode, radius_is_raw;
+    const void *radius;
+    float r_scalar, r_max, lo_cap, hi_cap;
+    int32_t policy;
+    float tau;
+    const float *u_flag;
+    ciar_quantify_out out;  // indexed by logical row
+};
+
+// Scratch of one verify launch, carved out of the caller's workspace.
+struct VerifyScratch {
+    int32_t *window_done;  // [windows] arrival counters, zero before the launch
+    int32_t *candidate;    // [rows] residual sample of each rejected row
+    uint8_t *accept;       // [rows] accept bits when the caller did not ask for them
+};
+
+struct VerifyArgs {
+    const void *draft, *target;
+    int64_t rows;  // logical rows, a multiple of the window
+    int64_t row_stride;
+    int32_t vocab, vb, n;
+    RowMap rm;
+    const int32_t *tokens;       // by physical row
+    const uint8_t *flag;         // by logical row
+    const float *draft_row_max;  // by logical row, nullable (then recomputed)
+    const float *draft_sum_exp;
+    const float *u_accept, *u_resample;  // by physical row
+    int32_t window, mode;
+    ciar_verify_out out;  // by logical row / logical window
+    VerifyScratch ws;
+};
+
+struct DecodeUpdateArgs {
+    ciar_decode_state st;
+    int32_t window, mode;
+    const int32_t *tokens;  // draft token pool
+    const uint8_t *flag;    // [requests * window] flags of this step
+    const int32_t *first_flag, *accepted_len, *resampled_token;  // [requests]
+};
+
+cudaError_t launch_quantify(const QuantifyArgs &a, int dtype, cudaStream_t stream);
+cudaError_t launch_verify(const VerifyArgs &a, int dtype, cudaStream_t stream);
+cudaError_t launch_decode_init(const ciar_decode_state &st, int32_t pos0, cudaStream_t stream);
+cudaError_t launch_decode_update(const DecodeUpdateArgs &a, cudaStream_t stream);
+
+int sm_count();       // SMs of the current device (cached per device)
+void count_launch();  // bumps the process-wide launch counter
+
+}  // namespace ciar

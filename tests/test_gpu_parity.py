@@ -1,0 +1,359 @@
+"""GPU parity: the CUDA path, called through the C ABI binding, against the CPU oracle on the
+same seeded input bytes.  Integer results bit-exact (near-tie rows reported separately), floating
+point within 1e-5 relative / 1e-7 absolute."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity_util as pu
+from paper_2603_25463_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ciar(ciar_lib):
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    return ciar_lib
+
+
+def _logits(rows, v, dtype, scale=3.0, seed=0):
+    g = torch.Generator().manual_seed(seed)
+    return (scale * torch.randn(rows, v, generator=g)).to(dtype)
+
+
+def _row_params(rows, seed=0, tau=None, **kw):
+    g = torch.Generator().manual_seed(seed + 77)
+    r = torch.rand(rows, generator=g) * 1.5
+    return oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=r, tau=1e-4 if tau is None else tau, **kw)
+
+
+# ---------------------------------------------------------------- quantify
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("v", [1, 2, 3, 7, 32, 33, 64, 1000, 2048, 16384])
+def test_quantify_small_shapes_dense(ciar, v, dtype):
+    rows = 24
+    stride = (v + 7) // 8 * 8
+    full = torch.full((rows, stride), float("nan"), dtype=dtype)
+    full[:, :v] = _logits(rows, v, dtype, seed=v)
+    logits = full[:, :v]  # row stride > vocab, padding holds NaN that must never be read
+    prm = _row_params(rows, seed=v)
+    dev = full.cuda()[:, :v]
+    ref, out, rep = pu.check_quantify(logits.contiguous(), prm, dense=True, logits_dev=dev)
+    assert rep.near_tie_flags <= 1
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("vb,n", [(0, 77), (3, 77), (5, 8), (8, 1), (13, 999), (1, 1030)])
+def test_quantify_unaligned_valid_slice(ciar, vb, n, dtype):
+    rows, vocab = 9, 1040
+    logits = _logits(rows, vocab, dtype, seed=vb + n)
+    logits[:, :vb] = float("nan")  # outside the slice: never read
+    logits[:, vb + n:] = float("inf")
+    pu.check_quantify(logits, _row_params(rows, seed=n), valid_begin=vb, valid_count=n, dense=True)
+
+
+@pytest.mark.parametrize("mode", ["scalar", "scalar_raw", "per_code", "per_code_raw"])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_quantify_radius_modes(ciar, mode, dtype):
+    rows, v = 16, 1500 if dtype == torch.float32 else 1504
+    logits = _logits(rows, v, dtype, scale=4.0, seed=3)
+    g = torch.Generator().manual_seed(5)
+    if mode == "scalar":
+        prm = oracle.IntervalParams(r_scalar=0.35, tau=1e-3)
+    elif mode == "scalar_raw":
+        prm = oracle.IntervalParams(r_scalar=-0.7, radius_is_raw=True, tau=1e-3)
+    elif mode == "per_code":
+        prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_CODE, radius=(torch.rand(rows, v, generator=g) * 2).to(dtype),
+                                    tau=1e-3)
+    else:
+        prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_CODE, radius_is_raw=True, r_max=1.5,
+                                    radius=torch.randn(rows, v, generator=g).to(dtype), tau=1e-3)
+    pu.check_quantify(logits, prm, dense=True)
+
+
+@pytest.mark.parametrize("r", [0.0, 1e-4, 0.05, 1.0, 5.0, 10.0, 40.0])
+def test_quantify_radius_extremes_and_closed_forms(ciar, r):
+    rows, v = 12, 4096
+    logits = _logits(rows, v, torch.float32, scale=6.0, seed=11)
+    ref, out, _ = pu.check_quantify(logits, oracle.IntervalParams(r_scalar=r, r_max=80.0, tau=1e-5), dense=True)
+    if r == 0.0:  # delta = 0.02 p: Omega = 0.02 exactly
+        np.testing.assert_allclose(out.omega.cpu().numpy(), 0.02, rtol=1e-6)
+
+
+def test_quantify_degenerate_rows(ciar):
+    v = 520
+    rows = []
+    one_hot = torch.full((v,), float("-inf")); one_hot[17] = 2.5; rows.append(one_hot)
+    rows.append(torch.full((v,), -0.75))  # constant row: Sigma = 0
+    near = torch.full((v,), -30.0); near[100] = 20.0; rows.append(near)  # p_max = 1 - 5e-20
+    two = torch.full((v,), float("-inf")); two[3] = 1.0; two[400] = 1.0; rows.append(two)
+    ties = torch.zeros(v); ties[40:44] = 5.0; rows.append(ties)  # arg-max tie -> lowest index
+    nan_row = torch.randn(v); nan_row[7] = float("nan"); rows.append(nan_row)
+    rows.append(torch.full((v,), float("-inf")))  # no finite code
+    inf_row = torch.randn(v); inf_row[9] = float("inf"); rows.append(inf_row)
+    big = torch.randn(v) * 1e4; rows.append(big)  # huge dynamic range
+    flat_small = torch.randn(v) * 1e-3; rows.append(flat_small)  # nearly uniform widths (low CV)
+    logits = torch.stack(rows)
+    for dtype in (torch.float32, torch.bfloat16):
+        for r in (0.0, 0.3, 2.0):
+            ref, out, _ = pu.check_quantify(logits.to(dtype), oracle.IntervalParams(r_scalar=r, tau=1e-4), dense=True)
+            st = out.row_status.cpu().numpy()
+            assert st[5] == oracle.ROW_NAN and st[6] == oracle.ROW_NO_FINITE and st[7] == oracle.ROW_NAN
+            assert out.flag.cpu().numpy()[5:8].all()
+            assert out.argmax.cpu().numpy()[4] == 40
+
+
+def test_quantify_policies(ciar):
+    rows, v = 64, 1024
+    logits = _logits(rows, v, torch.bfloat16, scale=2.0, seed=21)
+    base = oracle.quantify(logits, oracle.IntervalParams(r_scalar=0.5))
+    u = torch.rand(rows, generator=torch.Generator().manual_seed(1))
+    for policy, tau in ((oracle.POLICY_INTERVAL, float(np.median(base.score))),
+                        (oracle.POLICY_ENTROPY, float(np.median(base.entropy))),
+                        (oracle.POLICY_MAXPROB, float(np.median(base.p_max))),
+                        (oracle.POLICY_RANDOM, 0.4), (oracle.POLICY_ALL, 0.0)):
+        prm = oracle.IntervalParams(r_scalar=0.5, policy=policy, tau=tau, u_flag=u)
+        ref, out, rep = pu.check_quantify(logits, prm)
+        assert 0 < ref.flag.sum() <= rows
+
+
+def test_quantify_empty_and_optional_outputs(ciar):
+    empty = torch.empty((0, 64), dtype=torch.float32, device="cuda")
+    before = ciar.launch_count()
+    ciar.quantify(empty, ciar.IntervalParams(r_scalar=0.1), ciar.QuantifyOut.allocate(0, "cuda"))
+    assert ciar.launch_count() == before
+    logits = _logits(8, 256, torch.float32).cuda()
+    out = ciar.QuantifyOut(score=torch.empty(8, device="cuda"), flag=torch.empty(8, dtype=torch.uint8, device="cuda"))
+    ciar.quantify(logits, ciar.IntervalParams(r_scalar=0.1, tau=1e-4), out)
+    ref = oracle.quantify(logits.cpu(), oracle.IntervalParams(r_scalar=0.1, tau=1e-4))
+    pu.assert_close("score", out.score.cpu().numpy(), ref.score)
+
+
+def test_quantify_is_deterministic(ciar):
+    logits = _logits(64, 16384, torch.bfloat16, seed=5).cuda()
+    prm = ciar.IntervalParams(r_scalar=0.4, tau=1e-4)
+    a = ciar.QuantifyOut.allocate(64, "cuda")
+    b = ciar.QuantifyOut.allocate(64, "cuda")
+    ciar.quantify(logits, prm, a)
+    ciar.quantify(logits, prm, b)
+    torch.cuda.synchronize()
+    for name in pu.Q_FLOAT_FIELDS:
+        assert torch.equal(getattr(a, name), getattr(b, name)), name
+
+
+def test_binding_errors_are_loud(ciar):
+    logits = _logits(8, 256, torch.float32).cuda()
+    with pytest.raises(ciar.CiarError) as e:
+        ciar.quantify(logits.half(), ciar.IntervalParams(r_scalar=0.1), ciar.QuantifyOut.allocate(8, "cuda"))
+    assert e.value.status == 2
+    with pytest.raises(ciar.CiarError) as e:
+        ciar.quantify(logits[:, 1:], ciar.IntervalParams(r_scalar=0.1), ciar.QuantifyOut.allocate(8, "cuda"))
+    assert e.value.status == 3
+    with pytest.raises(ValueError):
+        ciar.quantify(logits.cpu(), ciar.IntervalParams(r_scalar=0.1), ciar.QuantifyOut.allocate(8, "cuda"))
+
+
+# ---------------------------------------------------------------- verify
+
+def _verify_case(rows, v, dtype, window, seed, sigma=0.7, scale=2.0):
+    g = torch.Generator().manual_seed(seed)
+    draft = (scale * torch.randn(rows, v, generator=g)).to(dtype)
+    target = (draft.float() + sigma * torch.randn(rows, v, generator=g)).to(dtype)
+    gum = -torch.log(-torch.log(torch.rand(rows, v, generator=g).clamp(1e-9, 1 - 1e-7)))
+    tokens = torch.argmax(draft.float() + gum, dim=1).to(torch.int32)
+    flag = (torch.rand(rows, generator=g) < 0.3).to(torch.uint8).numpy()
+    ua = torch.rand(rows, generator=g).numpy().astype(np.float32)
+    ur = torch.rand(rows, generator=g).numpy().astype(np.float32)
+    return draft, target, tokens.numpy(), flag, ua, ur
+
+
+@pytest.mark.parametrize("mode", [oracle.VERIFY_ANCHORED, oracle.VERIFY_PER_TOKEN, oracle.VERIFY_ALL])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("v,window", [(1, 1), (2, 2), (7, 4), (33, 8), (1000, 8), (2056, 16), (16384, 8)])
+def test_verify_small_shapes(ciar, v, window, dtype, mode):
+    rows = window * 12
+    draft, target, tok, flag, ua, ur = _verify_case(rows, v, dtype, window, seed=v * 7 + mode)
+    ref, out, rep = pu.check_verify(draft, target, tok, flag, ua, ur, window, mode)
+    assert rep.excluded_windows <= 2
+    if v >= 33 and mode == oracle.VERIFY_ALL:
+        assert (ref.resampled_token >= 0).any()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_verify_with_quantify_stats_and_slice(ciar, dtype):
+    rows, vocab, vb, n, window = 64, 2080, 37, 1999, 8
+    draft, target, tok, flag, ua, ur = _verify_case(rows, vocab, dtype, window, seed=99)
+    draft[:, :vb] = float("nan"); target[:, :vb] = float("nan")
+    draft[:, vb + n:] = 50.0; target[:, vb + n:] = 50.0
+    tok = np.clip(tok, vb, vb + n - 1).astype(np.int32)
+    tok[5] = 3  # a drafted code outside the valid slice has probability 0 under both models: rejected
+    flag[0] = 1
+    dd, td = draft.cuda(), target.cuda()
+    qo = ciar.QuantifyOut.allocate(rows, "cuda")
+    ciar.quantify(dd, ciar.IntervalParams(r_scalar=0.2, tau=1e-4), qo, vb, n)
+    ref, out, rep = pu.check_verify(draft, target, tok, flag, ua, ur, window, oracle.VERIFY_ANCHORED, vb, n,
+                                    draft_stats=(qo.row_max, qo.sum_exp), draft_dev=dd, target_dev=td)
+    assert ref.accept[5] == 0 and ref.p_draft_tok[5] == 0.0
+
+
+def test_verify_degenerate_rows(ciar):
+    v, window = 264, 4
+    draft, target, tok, flag, ua, ur = _verify_case(16, v, torch.float32, window, seed=4)
+    target[1] = draft[1]  # identical rows: always accepted
+    draft[2] = float("-inf"); draft[2, 5] = 0.0; target[2] = float("-inf"); target[2, 9] = 0.0; tok[2] = 5  # disjoint one-hots
+    ua[2] = 0.0
+    draft[6, 3] = float("nan")  # NaN draft row -> status, rejected, no token
+    target[9] = float("-inf")  # target without a finite code
+    tok[13] = v + 5  # token id out of range
+    tok[14] = -2
+    # identical distributions but the token has zero mass -> rejected with zero residual -> mode of q
+    draft[12] = target[12]; draft[12, 7] = float("-inf"); target[12, 7] = float("-inf"); tok[12] = 7
+    ref, out, rep = pu.check_verify(draft, target, tok, None, ua, ur, window, oracle.VERIFY_ALL)
+    assert ref.accept[1] == 1 and ref.accept[2] == 0
+    assert ref.resampled_token[0] >= 0
+    st = out.row_status.cpu().numpy()
+    assert st[6] & oracle.ROW_NAN and st[9] & oracle.ROW_NO_FINITE and st[13] & oracle.ROW_BAD_TOKEN and st[14]
+    assert out.resampled_token.cpu().numpy()[3] == int(torch.argmax(target[12]))
+
+
+def test_verify_endpoints_of_the_inverse_cdf(ciar):
+    rows, v, window = 32, 4096, 1
+    draft, target, tok, flag, ua, ur = _verify_case(rows, v, torch.bfloat16, window, seed=8, sigma=1.0)
+    ua[:] = 1 - 2.0 ** -24
+    p = torch.softmax(draft.double(), 1); q = torch.softmax(target.double(), 1)
+    tok = torch.argmin(q / p, dim=1).to(torch.int32).numpy()  # always rejected
+    for u in (0.0, 1 - 2.0 ** -24):
+        ur[:] = u
+        ref, out, rep = pu.check_verify(draft, target, tok, None, ua, ur, window, oracle.VERIFY_ALL)
+        assert (ref.accept == 0).all()
+
+
+def test_verify_errors(ciar):
+    draft, target, tok, flag, ua, ur = _verify_case(16, 64, torch.float32, 8, seed=1)
+    d, t = draft.cuda(), target.cuda()
+    args = lambda: (torch.as_tensor(tok).cuda(), torch.as_tensor(flag).cuda(), None, None,
+                    torch.as_tensor(ua).cuda(), torch.as_tensor(ur).cuda())
+    out = ciar.VerifyOut.allocate(16, 8, "cuda")
+    ws = ciar.alloc_workspace(16, 8, "cuda")
+    with pytest.raises(ciar.CiarError) as e:
+        ciar.verify(d, t, *args(), 5, ciar.VERIFY_ANCHORED, out, ws)
+    assert e.value.status == 1
+    with pytest.raises(ciar.CiarError) as e:
+        ciar.verify(d, t, *args(), 8, ciar.VERIFY_ANCHORED, out, ws[:16])
+    assert e.value.status == 4
+    ciar.verify(d, t, *args(), 8, ciar.VERIFY_ANCHORED, out, ws)  # the context is still healthy
+    torch.cuda.synchronize()
+
+
+# ---------------------------------------------------------------- the five workloads
+
+def _pipeline(ciar, wl, inp_cpu, inp_dev=None, per_code=False, threads=0):
+    """quantify -> verify on both sides (each side uses ITS OWN flags), reports near ties."""
+    dev = inp_dev if inp_dev is not None else None
+    dd = inp_cpu.draft.cuda() if dev is None else dev.draft
+    td = inp_cpu.target.cuda() if dev is None else dev.target
+    if per_code:
+        prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_CODE, radius=inp_cpu.radius_code, radius_is_raw=True,
+                                    tau=wl.tau)
+    else:
+        prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=inp_cpu.radius_row, tau=wl.tau)
+    ref_q, out_q, rep = pu.check_quantify(inp_cpu.draft, prm, wl.valid_begin, wl.n_valid, logits_dev=dd, threads=threads)
+    assert rep.near_tie_flags == 0  # tau sits in the gap between the two token classes
+    flags = ref_q.flag
+    assert np.array_equal(out_q.flag.cpu().numpy(), flags)
+    ref_v, out_v, rep_v = pu.check_verify(inp_cpu.draft, inp_cpu.target, inp_cpu.tokens.numpy(), flags,
+                                          inp_cpu.u_accept.numpy(), inp_cpu.u_resample.numpy(), wl.window,
+                                          oracle.VERIFY_ANCHORED, wl.valid_begin, wl.n_valid,
+                                          draft_stats=(out_q.row_max, out_q.sum_exp), draft_dev=dd, target_dev=td,
+                                          threads=threads)
+    return ref_q, ref_v, rep.merge(rep_v)
+
+
+def test_workload_llamagen256_full(ciar):
+    wl = synth.WORKLOADS["llamagen256"]
+    inp = synth.make_inputs(wl)
+    ref_q, ref_v, rep = _pipeline(ciar, wl, inp)
+    assert abs(ref_q.flag.mean() - 0.30) < 0.02
+    assert rep.excluded_windows <= 2
+
+
+def test_workload_llamagen384_full(ciar):
+    wl = synth.WORKLOADS["llamagen384"]
+    inp = synth.make_inputs(wl)
+    ref_q, ref_v, rep = _pipeline(ciar, wl, inp)
+    assert abs(ref_q.flag.mean() - 0.30) < 0.01
+    assert rep.excluded_windows <= 0.05 * rep.windows
+
+
+def test_workload_llamagen384_per_code_radius(ciar):
+    wl = synth.WORKLOADS["llamagen384"].scaled(images=2)
+    inp = synth.make_inputs(wl, per_code_radius=True)
+    _pipeline(ciar, wl, inp, per_code=True)
+
+
+def test_workload_anole_full(ciar):
+    wl = synth.WORKLOADS["anole"]
+    inp = synth.make_inputs(wl)
+    ref_q, ref_v, rep = _pipeline(ciar, wl, inp)
+    assert abs(ref_q.flag.mean() - 0.30) < 0.01
+    assert (ref_q.argmax >= wl.valid_begin).all() and (ref_q.argmax < wl.valid_begin + wl.n_valid).all()
+
+
+def test_workload_largevocab_sample(ciar):
+    """The stress workload at full width (V = 2^18) on a bounded number of rows."""
+    wl = synth.WORKLOADS["largevocab"].scaled(images=1, grid_h=8, grid_w=16)
+    inp = synth.make_inputs(wl)
+    ref_q, ref_v, rep = _pipeline(ciar, wl, inp)
+    assert ref_q.flag.any() and not ref_q.flag.all()
+
+
+# ---------------------------------------------------------------- decode loop
+
+def _decode_compare(ciar, wl, mode=oracle.VERIFY_ANCHORED, pos0=0, max_steps=None):
+    inp = synth.make_inputs(wl)
+    seq, req = wl.tokens_per_image, wl.images
+    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
+    ost = oracle.DecodeState(req, seq, pos0)
+    gst = ciar.DecodeState.allocate(req, seq, "cuda")
+    ciar.decode_init(gst, pos0)
+    dd, td = inp.draft.cuda(), inp.target.cuda()
+    tok, ua, ur = inp.tokens.cuda(), inp.u_accept.cuda(), inp.u_resample.cuda()
+    gp = pu.to_ciar_params(prm, "cuda")
+    ws = ciar.alloc_workspace(req * wl.window, wl.window, "cuda")
+    steps = 0
+    while (ost.pos < seq).any():
+        oracle.decode_step(ost, inp.draft, inp.target, inp.tokens, inp.u_accept, inp.u_resample, prm, wl.window, mode,
+                           wl.valid_begin, wl.n_valid)
+        ciar.decode_step(gst, dd, td, tok, ua, ur, gp, wl.window, mode, ws, wl.valid_begin, wl.n_valid)
+        steps += 1
+        if ost.min_margin.min() < pu.NEAR_TIE:
+            pytest.skip("a near-tie decision occurred; trajectories may legitimately diverge")
+        assert np.array_equal(gst.pos.cpu().numpy(), ost.pos), "pos after step %d" % steps
+        if max_steps and steps >= max_steps:
+            break
+    torch.cuda.synchronize()
+    assert np.array_equal(gst.tokens_out.cpu().numpy(), ost.tokens_out)
+    assert np.array_equal(gst.counters.cpu().numpy(), ost.counters)
+    return steps, ost
+
+
+@pytest.mark.parametrize("mode", [oracle.VERIFY_ANCHORED, oracle.VERIFY_PER_TOKEN, oracle.VERIFY_ALL])
+def test_decode_loop_small(ciar, mode):
+    wl = synth.Workload("dec", 6, 5, 8, 512, "bf16", 8, 0.5, seed=13, decode=True, tau=2e-3)
+    steps, ost = _decode_compare(ciar, wl, mode)
+    assert (ost.pos == wl.tokens_per_image).all() and (ost.tokens_out >= 0).all()
+
+
+def test_decode_loop_prefix_and_ragged_tail(ciar):
+    wl = synth.Workload("dec2", 5, 3, 9, 1000, "f32", 8, 0.5, seed=14, decode=True, tau=1e-3)  # 27 tokens: ragged windows
+    _decode_compare(ciar, wl, pos0=2)
+
+
+def test_decode_workload_shape_few_steps(ciar):
+    """The serving workload's per-step shape (V = 16384, window 8) on fewer requests."""
+    wl = synth.WORKLOADS["decode"].scaled(images=16, grid_h=8, grid_w=8)
+    _decode_compare(ciar, wl)
