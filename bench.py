@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the CIAR hot path: tokens/s quantified + verified on synthetic LlamaGen-384-like
+logits (16 images x 24x24 tokens, V = 16384, bf16, draft window 16).
+
+One "step" is one pass of the whole path over the batch: ciar_quantify on every row, then
+ciar_verify (Algorithm 1's anchored windows) with the flags and softmax statistics quantify
+produced.  `value` times K steps with the inputs resident in HBM; `e2e` times the same calls
+with the step's inputs copied from pinned host memory and the results copied back inside the
+timed region.  `--impl reference` times the CPU oracle on a bounded sample of the same workload.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+Multi-GPU: launched by torchrun, one rank per GPU; every rank processes its own batch (weak
+scaling), no data-path collective; time = max over ranks.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2603_25463_b200 import synth
+
+METRIC = "tokens/s quantified+verified"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi polled in the background while the timed region runs (read-only)."""
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        self.path = "/tmp/ciar_clocks_%d_%d.csv" % (os.getpid(), device_index)
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            sel = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            sel = str(device_index)
+        self.cmd = ["nvidia-smi", "-i", sel, "--query-gpu=" + CLOCK_QUERY, "--format=csv,noheader,nounits", "-lms", "100"]
+
+    def start(self):
+        try:
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(self.cmd, stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            res.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return res
+
+
+def dist_setup(n_gpus):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(x: float, world: int) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+class Step:
+    """The hot path on one resident batch: quantify -> verify through the C ABI binding."""
+
+    def __init__(self, ciar, wl, inp):
+        self.ciar, self.wl = ciar, wl
+        dev = inp.draft.device
+        self.draft, self.target = inp.draft, inp.target
+        self.tokens, self.ua, self.ur = inp.tokens, inp.u_accept, inp.u_resample
+        self.params = ciar.IntervalParams(radius_mode=ciar.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
+        rows = inp.draft.shape[0]
+        self.rows = rows
+        self.qout = ciar.QuantifyOut.allocate(rows, dev)
+        self.vout = ciar.VerifyOut.allocate(rows, wl.window, dev)
+        self.ws = ciar.alloc_workspace(rows, wl.window, dev)
+
+    def quantify(self):
+        self.ciar.quantify(self.draft, self.params, self.qout, self.wl.valid_begin, self.wl.n_valid)
+
+    def verify(self):
+        self.ciar.verify(self.draft, self.target, self.tokens, self.qout.flag, self.qout.row_max, self.qout.sum_exp,
+                         self.ua, self.ur, self.wl.window, self.ciar.VERIFY_ANCHORED, self.vout, self.ws,
+                         self.wl.valid_begin, self.wl.n_valid)
+
+    def __call__(self):
+        self.quantify()
+        self.verify()
+
+    def traffic_model(self):
+        """Rows the method has to touch in this batch: (sent rows, resampled rows, flagged fraction)."""
+        f = self.vout.first_flag.cpu().numpy().astype(np.int64)
+        a = self.vout.accepted_len.cpu().numpy().astype(np.int64)
+        w = self.wl.window
+        sent = int((w - f).sum())
+        resampled = int((a < w).sum())
+        flagged = float(self.qout.flag.float().mean().item())
+        return sent, resampled, flagged
+
+
+def run_ours(args):
+    from paper_2603_25463_b200 import ciar
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local if world > 1 else 0)
+    wl = synth.WORKLOADS[args.workload]
+    wl = wl.scaled(seed=wl.seed + 101 * rank)  # every rank draws its own batch (weak scaling)
+    inp = synth.make_inputs(wl, device=dev)
+    step = Step(ciar, wl, inp)
+    rows = step.rows
+    row_bytes = wl.n_valid * wl.elem_bytes
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    sent, resampled, flagged = step.traffic_model()
+
+    # ---- device-resident timing: K steps, events around every kernel of every step
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    sampler = ClockSampler(dev.index or 0)
+    launches0 = ciar.launch_count()
+    sampler.start()
+    barrier(world)
+    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for k in range(K):
+        ev[k][0].record()
+        step.quantify()
+        ev[k][1].record()
+        step.verify()
+        ev[k][2].record()
+    t_end.record()
+    barrier(world)
+    clocks = sampler.stop()
+    launches = ciar.launch_count() - launches0
+    total_ms = max_over_ranks(t_start.elapsed_time(t_end), world)
+    q_ms = float(np.mean([ev[k][0].elapsed_time(ev[k][1]) for k in range(K)]))
+    v_ms = float(np.mean([ev[k][1].elapsed_time(ev[k][2]) for k in range(K)]))
+    ms_per_step = total_ms / K
+    value = world * rows * K / (total_ms * 1e-3)
+
+    # ---- end to end: inputs start in pinned host memory, results end in host memory
+    e2e = None
+    if not args.no_e2e:
+        hd, ht = inp.draft.cpu().pin_memory(), inp.target.cpu().pin_memory()
+        htok, hua, hur, hrad = (x.cpu().pin_memory() for x in (inp.tokens, inp.u_accept, inp.u_resample, inp.radius_row))
+        res_dev = [step.qout.flag, step.qout.score, step.vout.accept, step.vout.accepted_len, step.vout.resampled_token,
+                   step.vout.first_flag]
+        res_host = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in res_dev]
+        ins = [(step.draft, hd), (step.target, ht), (step.tokens, htok), (step.ua, hua), (step.ur, hur),
+               (step.params.radius, hrad)]
+        h2d = sum(h.numel() * h.element_size() for _, h in ins)
+        d2h = sum(h.numel() * h.element_size() for h in res_host)
+
+        def e2e_step():
+            for d, h in ins:
+                d.copy_(h, non_blocking=True)
+            step()
+            for d, h in zip(res_dev, res_host):
+                h.copy_(d, non_blocking=True)
+        Ke = max(3, min(K, args.e2e_steps))
+        for _ in range(3):
+            e2e_step()
+        barrier(world)
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for _ in range(Ke):
+            e2e_step()
+        e.record()
+        barrier(world)
+        e_ms = max_over_ranks(s.elapsed_time(e), world)
+        e2e = {"value": world * rows * Ke / (e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "steps": Ke, "ms_per_step": e_ms / Ke}
+
+    if rank != 0:
+        return
+    peak, peak_kind = measured_peak()
+    q_bytes = rows * row_bytes + rows * 48
+    v_bytes = sent * row_bytes + resampled * 2 * row_bytes + rows * 16 + (rows // wl.window) * 16
+    q_gbs = q_bytes / (q_ms * 1e-3) / 1e9
+    v_gbs = v_bytes / (v_ms * 1e-3) / 1e9
+    dominant = "quantify_kernel" if q_ms >= v_ms else "verify_kernel"
+    dom_gbs = q_gbs if q_ms >= v_ms else v_gbs
+    traffic = load_traffic(dominant, args.workload)
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
+                "frac": dom_gbs / peak, "peak_kind": "of " + peak_kind, "traffic": traffic,
+                "frac_of_nominal_8TBs": dom_gbs / NOMINAL_HBM_GBS,
+                "kernels": {"quantify_kernel": {"ms": q_ms, "algorithmic_bytes": int(q_bytes), "GB/s": q_gbs,
+                                                "frac": q_gbs / peak},
+                            "verify_kernel": {"ms": v_ms, "algorithmic_bytes": int(v_bytes), "GB/s": v_gbs,
+                                              "frac": v_gbs / peak}},
+                "step_GB/s": (q_bytes + v_bytes) / (ms_per_step * 1e-3) / 1e9}
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_oracle_baseline(synth.WORKLOADS[args.workload], sample_rows=args.cpu_rows)
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "rows_per_gpu": rows, "vocab": wl.vocab, "valid_codes": wl.n_valid,
+                   "logits": wl.dtype, "window": wl.window, "verify_mode": "anchored", "radius": "per_row",
+                   "tau": wl.tau, "l2": "inputs (%.0f MB) larger than L2; no flush" % (2 * rows * row_bytes / 1e6)},
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+        "cloud_flag_fraction": flagged, "sent_fraction": sent / rows, "resampled_windows": resampled,
+    }
+    print(json.dumps(line))
+
+
+def load_traffic(kernel, workload):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if one exists."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f).get(workload, {}).get(kernel)
+    except Exception:
+        return None
+
+
+def cpu_oracle_baseline(wl, sample_rows, threads=0):
+    """The CPU oracle, as it stands, timed on a bounded sample of the same workload (whole images)."""
+    import oracle
+    inp = synth.make_inputs(wl, device="cpu", row_limit=sample_rows)
+    rows = inp.draft.shape[0]
+    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
+    oracle.quantify(inp.draft[:wl.window], prm, wl.valid_begin, wl.n_valid)  # load the library
+    t0 = time.perf_counter()
+    q = oracle.quantify(inp.draft, prm, wl.valid_begin, wl.n_valid, threads=threads)
+    oracle.verify(inp.draft, inp.target, inp.tokens, q.flag, inp.u_accept, inp.u_resample, wl.window,
+                  oracle.VERIFY_ANCHORED, wl.valid_begin, wl.n_valid, threads=threads)
+    dt = time.perf_counter() - t0
+    cores = threads or oracle.max_threads()
+    return {"value": rows / dt, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "sample": "first %d rows of %s (quantify + verify), %.2f s wall" % (rows, wl.name, dt)}
+
+
+def run_reference(args):
+    """The base contract's reference arm: here the CPU oracle on host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    wl = synth.WORKLOADS[args.workload]
+    steps = max(1, min(args.steps, 20))
+    warm = max(1, min(args.warmup, 2))
+    inp = synth.make_inputs(wl, device="cpu", row_limit=args.cpu_rows)
+    rows = inp.draft.shape[0]
+    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
+
+    def one():
+        q = oracle.quantify(inp.draft, prm, wl.valid_begin, wl.n_valid)
+        oracle.verify(inp.draft, inp.target, inp.tokens, q.flag, inp.u_accept, inp.u_resample, wl.window,
+                      oracle.VERIFY_ANCHORED, wl.valid_begin, wl.n_valid)
+    for _ in range(warm):
+        one()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    dt = time.perf_counter() - t0
+    value = rows * steps / dt
+    cores = oracle.max_threads()
+    sample = "each step = first %d rows of %s through the CPU oracle (quantify + verify)" % (rows, wl.name)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": steps,
+        "warmup": warm, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "rows_per_step": rows, "vocab": wl.vocab, "valid_codes": wl.n_valid,
+                   "logits": wl.dtype, "window": wl.window, "verify_mode": "anchored", "radius": "per_row"},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llamagen384", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--cpu-rows", type=int, default=9216, help="rows of the CPU oracle's bounded sample")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CIAR path has no CPU fallback "
+                         "(use --impl reference for the CPU oracle)")
+    run_ours(args)
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

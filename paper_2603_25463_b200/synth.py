@@ -175,8 +175,10 @@ def make_inputs(wl: Workload, device="cpu", per_code_radius: bool = False, row_l
     """Generate a workload's tensors on ``device``.  ``row_limit`` keeps only the first rows
     (a whole number of windows) -- used for bounded samples of a large workload."""
     dev = torch.device(device)
-    rows = wl.rows if row_limit is None else min(wl.rows, row_limit)
-    rows -= rows % wl.window
+    rows = wl.rows
+    if row_limit is not None:
+        rows = min(rows, row_limit)
+        rows -= rows % wl.window
     gen = torch.Generator(device=dev)
     gen.manual_seed(7919 * wl.seed + 3)
     boundary = blob_boundary_mask(wl).reshape(-1)[:rows].to(dev)

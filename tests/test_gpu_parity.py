@@ -177,7 +177,10 @@ def _verify_case(rows, v, dtype, window, seed, sigma=0.7, scale=2.0):
 def test_verify_small_shapes(ciar, v, window, dtype, mode):
     rows = window * 12
     draft, target, tok, flag, ua, ur = _verify_case(rows, v, dtype, window, seed=v * 7 + mode)
-    ref, out, rep = pu.check_verify(draft, target, tok, flag, ua, ur, window, mode)
+    stride = (v + 7) // 8 * 8  # device rows padded to a 16-byte multiple; the padding is never read
+    pad = lambda t: torch.cat([t, torch.full((rows, stride - v), float("nan"), dtype=dtype)], 1).cuda()[:, :v]
+    ref, out, rep = pu.check_verify(draft, target, tok, flag, ua, ur, window, mode,
+                                    draft_dev=pad(draft), target_dev=pad(target))
     assert rep.excluded_windows <= 2
     if v >= 33 and mode == oracle.VERIFY_ALL:
         assert (ref.resampled_token >= 0).any()
