@@ -60,8 +60,9 @@ enum { CIAR_POLICY_INTERVAL = 0, CIAR_POLICY_ENTROPY = 1, CIAR_POLICY_MAXPROB = 
    the first flagged token and runs to the end of the window.  PER_TOKEN tests flagged rows only.
    ALL tests every row. */
 enum { CIAR_VERIFY_ANCHORED = 0, CIAR_VERIFY_PER_TOKEN = 1, CIAR_VERIFY_ALL = 2 };
-/* row_status bits */
-enum { CIAR_ROW_NAN = 1, CIAR_ROW_NO_FINITE = 2, CIAR_ROW_BAD_TOKEN = 4 };
+/* row_status bits.  TIMEOUT: the device gave up waiting for the row's data to arrive on chip (a
+   bounded wait ran out; never expected in normal operation); the row's results are unusable. */
+enum { CIAR_ROW_NAN = 1, CIAR_ROW_NO_FINITE = 2, CIAR_ROW_BAD_TOKEN = 4, CIAR_ROW_TIMEOUT = 8 };
 
 #define CIAR_MAX_WINDOW 64
 

@@ -52,6 +52,9 @@ struct DecodeUpdateArgs {
 };
 
 cudaError_t launch_quantify(const QuantifyArgs &a, int dtype, cudaStream_t stream);
+// The streaming (TMA ring) quantifier and the test that says whether it covers a call.
+bool quantify_stream_eligible(const QuantifyArgs &a, int dtype);
+cudaError_t launch_quantify_stream(const QuantifyArgs &a, int dtype, cudaStream_t stream);
 cudaError_t launch_verify(const VerifyArgs &a, int dtype, cudaStream_t stream);
 cudaError_t launch_decode_init(const ciar_decode_state &st, int32_t pos0, cudaStream_t stream);
 cudaError_t launch_decode_update(const DecodeUpdateArgs &a, cudaStream_t stream);
