@@ -28,25 +28,40 @@ constexpr long long kDrainCycles = 20000000ll;                 // bound of each 
 constexpr float kLogitFloor = -1.329227995784916e36f;
 constexpr uint32_t kLogitFloorBf16x2 = 0xFB80FB80u;
 
-// Interval constants of one row.  With x = softmax probability and s = 1 - x the raw bounds are
-//   p^l = a1 x / den_l,  p^u - p^l = kd x s / (den_l den_u),  den_l = a1 + b1 s,  den_u = a1 + b1 x,
-// where (a1, b1, kd) = (1, beta, beta (2 + beta)) for beta = e^r - 1 <= 1 and (1 / beta, 1, 1 + 2 / beta)
-// otherwise (the second form keeps every term in range for radii up to 80).
+// Interval constants of one row, worked out by one consumer thread per row.
+//
+// With x = softmax probability, s = 1 - x and beta = e^r - 1 the raw InterFuse bounds are
+//   p^l = x / (1 + beta s),   p^u = (1 + beta) x / (1 + beta x),
+//   p^u - p^l = beta (2 + beta) x s / ((1 + beta s)(1 + beta x)).
+// Rows with r <= 1 take the "series" route: every code with x below theta = 2^-8 / (1 + beta) enters
+// only through the power sums of (e - c0) up to the fourth (c0 = Z / n), from which the finalizer
+// rebuilds the sums of p^l, of the widths and of their squares by a fourth-order Taylor expansion
+// about x0 = 1 / n (terms beyond it are below 1e-7 of the result); the few codes above theta are
+// clamped to it in the power sums, listed, and put back exactly.  Rows with r > 1 take the
+// "direct" route: both bounds of every code from the formulas above, in the scaled form
+//   den_l = a1 + b1 s, den_u = a1 + b1 x, (a1, b1) = (1, beta) or (1 / beta, 1) for beta > 1,
+// which keeps every term in range for radii up to 80.
 struct RowConst {
-    float a1, b1;
-    float pl0, dd0;  // the two raw terms at x = 1 / n: the sums are accumulated about these values
-    float r;         // clamped radius; NaN marks an unusable radius
+    float rho;       // radius as stored (before Softplus when raw); NaN marks an unusable radius
+    float r;         // clamped radius
+    float theta_p;   // series route: probability above which a code is treated exactly
+    float a1, b1;    // direct route
+    float pl0, dd0;  // direct route: the two raw terms at x = 1 / n, about which its sums are taken
+    int series;
     int big;
 };
 
+constexpr int kListCap = 704;  // > 256 (1 + beta) for r <= 1: more codes than that cannot exceed theta
+
 struct RowInfo {
     long long lr, pr;
-    float m, e0;  // row maximum; the exponential of a code equal to it, as the consumers computed it
+    float m, e0;   // row maximum; the exponential of a code equal to it, as the consumers computed it
+    float c0, th;  // series route: centre of the power sums and clamp level, in units of exp(c - m)
     int argmin, nmax;
     int status;  // CIAR_ROW_* bits found by the consumers (0 = a regular row)
     int cmd;     // 0 = finalize this row, 1 = no more rows
     RowConst rc;
-    float2 zt[kQWarps];  // per-warp sums of exp and of exp * exponent
+    float2 zt[kQWarps];  // per-warp sums of exp (maxima left out) and of exp * exponent
 };
 
 struct QShared {
@@ -54,22 +69,26 @@ struct QShared {
     float wmax[kQWarps];
     float wz[kQWarps];
     RowConst rc[2];
-    int argmin, nmax;  // lowest index holding the row maximum, number of codes equal to it
+    int argmin, nmax;  // lowest index holding the row maximum, number of codes whose exponential equals e0
     int bad_nan, bad_finite;
     int abort;
+    int nlist;  // codes above theta in the row being swept (reset by the finalizer when it has read them)
     RowInfo info;
     float part[5][kQConsumers];
+    float list[kListCap];
 };
 
 __device__ __forceinline__ RowConst make_row_const(float rho, int raw, float r_max, int n)
 {
     RowConst k;
+    k.rho = rho;
     float r = rho;
     if (raw) r = (rho > 0.f) ? rho + log1pf(expf(-rho)) : log1pf(expf(rho));  // Softplus, beta = 1
-    r = fminf(r, r_max);                                                     // NaN stays NaN
-    if (!(rho == rho)) r = rho;
+    r = fminf(r, r_max);
     k.r = r;
     const float beta = expm1f(r);
+    k.series = r <= 1.0f;
+    k.theta_p = 0.00390625f / (1.0f + beta);
     k.big = beta > 1.0f;
     if (k.big) {
         k.a1 = 1.0f / beta;
@@ -210,64 +229,101 @@ __device__ __forceinline__ void write_unusable(const ciar_quantify_out &o, long 
     if (o.row_status) o.row_status[lr] = (uint8_t)status;
 }
 
-// One row's outputs from its reduced sums (normalisation step, Omega, Sigma, U, entropy, flag).
-__device__ __forceinline__ void finalize_one(const QuantifyArgs &a, const double (&s)[5], double zr, double tr,
-                                             long long lr, long long pr, float m, int argmin, int status,
-                                             const RowConst &rc)
+// What the consumers hand over for one row, reduced over the CTA (lane 0 of the finalizer).
+struct RowSums {
+    double s[5];    // series route: s[0..2] = sums of (e - c0)^2, ^3, ^4; direct route: the five centred sums
+    double zpart;   // sum of exp(c - m) without the maxima
+    double tr;      // sum of exp * exponent
+    double excess;  // series route: sum over listed codes of (e - clamp level)
+};
+
+// Omega, Sigma and the raw bound sums of a series-route row.  Listed codes are handled by all lanes.
+__device__ __forceinline__ void series_sums(const QuantifyArgs &a, const QShared &sh, const RowSums &rs, double beta,
+                                            float e0f, int nmax, float c0f, float thf, int nlist, float e_first, int lane,
+                                            double &S_lo, double &S_up, double &omega, double &sigma)
 {
-    const ciar_quantify_out &o = a.out;
-    if (status) {
-        write_unusable(o, lr, status);
-        return;
-    }
     const double nn = (double)a.n;
-    const double P1 = s[0], D1 = s[1], PP = s[2], PD = s[3], DD = s[4];
+    const double e0 = (double)e0f, zd = rs.zpart + (double)nmax * e0;  // the row's sum of exponentials
+    const double invz = 1.0 / zd;
+    const double b = 1.0 + beta, kap = beta * (2.0 + beta);
+    const double x0 = (double)c0f * invz, hth = ((double)thf - (double)c0f) * invz;
+    const double iz2 = invz * invz;
+    const double H1 = (zd - rs.excess - nn * (double)c0f) * invz;  // sum of (clamped x - x0)
+    const double H2 = rs.s[0] * iz2, H3 = rs.s[1] * iz2 * invz, H4 = rs.s[2] * iz2 * iz2;
+    // Taylor coefficients about x0 of p^l(x) = x / (b - beta x) and p^u(x) = b x / (1 + beta x)
+    const double u = b - beta * x0, v = 1.0 + beta * x0;
+    const double iuv = 1.0 / (u * v), iu = v * iuv, iv = u * iuv;
+    const double rl = beta * iu, ru = -beta * iv;
+    const double PL0 = x0 * iu, PL1 = b * iu * iu, PL2 = PL1 * rl, PL3 = PL2 * rl, PL4 = PL3 * rl;
+    const double PU1 = b * iv * iv, PU2 = PU1 * ru, PU3 = PU2 * ru, PU4 = PU3 * ru;
+    const double DD0 = kap * x0 * (1.0 - x0) * iuv;                        // p^u - p^l at x0, no cancellation
+    const double DD1 = b * beta * (1.0 - 2.0 * x0) * (u + v) * iuv * iuv;  // PU1 - PL1, no cancellation
+    const double DD2 = PU2 - PL2, DD3 = PU3 - PL3, DD4 = PU4 - PL4;
+    const double h2 = hth * hth, h3 = h2 * hth, h4 = h2 * h2;
+    const double pl_th = PL0 + PL1 * hth + PL2 * h2 + PL3 * h3 + PL4 * h4;  // what a clamped code contributed
+    const double dd_th = DD0 + DD1 * hth + DD2 * h2 + DD3 * h3 + DD4 * h4;
+    // listed codes, exactly: first their share of the bound sums
+    double bl = 0.0, dl = 0.0;
+    for (int i = lane; i < nlist; i += 32) {
+        const double e = i < 32 ? (double)e_first : (double)sh.list[i];
+        const double x = e * invz;
+        const double sx = (e == e0 ? rs.zpart + (double)(nmax - 1) * e0 : zd - e) * invz;  // 1 - x from the other codes
+        const double den = 1.0 / ((1.0 + beta * sx) * (1.0 + beta * x));
+        bl += x * (1.0 + beta * x) * den - pl_th;
+        dl += kap * x * sx * den - dd_th;
+    }
+    bl = warp_sum_d(bl);
+    dl = warp_sum_d(dl);
+    const double B = nn * PL0 + PL1 * H1 + PL2 * H2 + PL3 * H3 + PL4 * H4 + bl;  // sum of raw lower bounds
+    const double A = nn * DD0 + DD1 * H1 + DD2 * H2 + DD3 * H3 + DD4 * H4 + dl;  // sum of raw widths
+    S_lo = B;
+    S_up = A + B;
+    double k_lo = 1.0, k_up = 1.0;
+    if (S_lo > 0.0 && (double)a.lo_cap / S_lo < 1.0) k_lo = (double)a.lo_cap / S_lo;
+    if (S_up > 0.0 && (double)a.hi_cap / S_up > 1.0) k_up = (double)a.hi_cap / S_up;
+    const double g = k_up - k_lo;  // delta = k_up (p^u - p^l) + g p^l
+    omega = k_up * A + g * B;
+    const double mu = omega / nn;
+    const double E0 = k_up * DD0 + g * PL0 - mu, E1 = k_up * DD1 + g * PL1, E2 = k_up * DD2 + g * PL2,
+                 E3 = k_up * DD3 + g * PL3, E4 = k_up * DD4 + g * PL4;
+    const double q11 = E1 * E1, q12 = 2.0 * E1 * E2, q22 = 2.0 * E1 * E3 + E2 * E2;
+    double ss = nn * E0 * E0 + 2.0 * E0 * (E1 * H1 + E2 * H2 + E3 * H3 + E4 * H4) + q11 * H2 + q12 * H3 + q22 * H4;
+    const double sq_th = E0 * E0 + 2.0 * E0 * (E1 * hth + E2 * h2 + E3 * h3 + E4 * h4) + q11 * h2 + q12 * h3 + q22 * h4;
+    double sl = 0.0;
+    for (int i = lane; i < nlist; i += 32) {
+        const double e = i < 32 ? (double)e_first : (double)sh.list[i];
+        const double x = e * invz;
+        const double sx = (e == e0 ? rs.zpart + (double)(nmax - 1) * e0 : zd - e) * invz;
+        const double den = 1.0 / ((1.0 + beta * sx) * (1.0 + beta * x));
+        const double dev = k_up * (kap * x * sx * den) + g * (x * (1.0 + beta * x) * den) - mu;
+        sl += dev * dev - sq_th;
+    }
+    ss += warp_sum_d(sl);
+    sigma = sqrt((ss > 0.0 ? ss : 0.0) / nn);
+}
+
+// Omega, Sigma and the raw bound sums of a direct-route row (lane 0 only needs them).
+__device__ __forceinline__ void direct_sums(const QuantifyArgs &a, const RowSums &rs, const RowConst &rc, double &S_lo,
+                                            double &S_up, double &omega, double &sigma)
+{
+    const double nn = (double)a.n;
+    const double P1 = rs.s[0], D1 = rs.s[1], PP = rs.s[2], PD = rs.s[3], DD = rs.s[4];
     const double a1 = (double)rc.a1, b1 = (double)rc.b1;
     const double kd = rc.big ? 1.0 + 2.0 * a1 : b1 * (2.0 + b1);
-    const double B = nn * (double)rc.pl0 + P1;       // sum of the raw lower bounds
+    const double B = nn * (double)rc.pl0 + P1;  // sum of the raw lower bounds
     const double Dsum = nn * (double)rc.dd0 + D1;
-    const double A = kd * Dsum;                      // sum of the raw widths
-    const double S_lo = B, S_up = A + B;
+    const double A = kd * Dsum;  // sum of the raw widths
+    S_lo = B;
+    S_up = A + B;
     double k_lo = 1.0, k_up = 1.0;
     if (S_lo > 0.0 && (double)a.lo_cap / S_lo < 1.0) k_lo = (double)a.lo_cap / S_lo;
     if (S_up > 0.0 && (double)a.hi_cap / S_up > 1.0) k_up = (double)a.hi_cap / S_up;
     // delta_i = k_up d_i + (k_up - k_lo) p^l_i = c1 dd_i + c2 pl_i
     const double c1 = k_up * kd, c2 = k_up - k_lo;
-    const double omega = c1 * Dsum + c2 * B;
+    omega = c1 * Dsum + c2 * B;
     const double lin = c1 * D1 + c2 * P1;
-    double ss = c1 * c1 * DD + 2.0 * c1 * c2 * PD + c2 * c2 * PP - lin * lin / nn;
-    if (!(ss > 0.0)) ss = 0.0;
-    const double sigma = sqrt(ss / nn);
-    const double score = omega * sigma;
-    // exponent actually used: c * log2e_f - m2 = (c - m) * log2e_f + off with off = m * log2e_f - m2
-    const double off = (double)m * (double)kLog2e - (double)(m * kLog2e);
-    const double unscale = exp2(-off);
-    const double z = zr * unscale;
-    const double t = tr * unscale - off * z;
-    const double lnz = log(z);
-    const double entropy = lnz - kLn2D * t / z;
-    const double p_max = 1.0 / z;
-    int fl;
-    switch (a.policy) {
-    case CIAR_POLICY_INTERVAL: fl = score > (double)a.tau; break;
-    case CIAR_POLICY_ENTROPY: fl = entropy > (double)a.tau; break;
-    case CIAR_POLICY_MAXPROB: fl = p_max < (double)a.tau; break;
-    case CIAR_POLICY_RANDOM: fl = a.u_flag[pr] < a.tau; break;
-    default: fl = 1; break;
-    }
-    if (o.row_max) o.row_max[lr] = m;
-    if (o.sum_exp) o.sum_exp[lr] = (float)z;
-    if (o.lse) o.lse[lr] = (float)((double)m + lnz);
-    if (o.p_max) o.p_max[lr] = (float)p_max;
-    if (o.entropy) o.entropy[lr] = (float)entropy;
-    if (o.S_lo) o.S_lo[lr] = (float)S_lo;
-    if (o.S_up) o.S_up[lr] = (float)S_up;
-    if (o.omega) o.omega[lr] = (float)omega;
-    if (o.sigma) o.sigma[lr] = (float)sigma;
-    if (o.score) o.score[lr] = (float)score;
-    if (o.argmax) o.argmax[lr] = argmin + a.vb;
-    if (o.flag) o.flag[lr] = (uint8_t)fl;
-    if (o.row_status) o.row_status[lr] = 0;
+    const double ss = c1 * c1 * DD + 2.0 * c1 * c2 * PD + c2 * c2 * PP - lin * lin / nn;
+    sigma = sqrt((ss > 0.0 ? ss : 0.0) / nn);
 }
 
 // The finalizer warp: takes the per-thread partial sums of one row from the hand-off buffer,
@@ -275,41 +331,118 @@ __device__ __forceinline__ void finalize_one(const QuantifyArgs &a, const double
 // Sigma, U, entropy, the flag).
 __device__ __noinline__ void finalize_rows(const QuantifyArgs &a, QShared &sh, int lane)
 {
+    const ciar_quantify_out &o = a.out;
+    float beta_key = __int_as_float(0x7fc00000);  // stored radius whose e^r - 1 is cached in beta_val
+    double beta_val = 0.0;
     named_bar_arrive(kBarFree, kQBlock);
     for (;;) {
         named_bar_sync(kBarFull, kQBlock);
         if (sh.info.cmd) break;
-        double s[5];
+        const RowConst rc = sh.info.rc;
+        const int status = sh.info.status;
+        const int nk = rc.series ? 3 : 5;
+        RowSums rs;
 #pragma unroll
         for (int k = 0; k < 5; ++k) {
             double acc = 0.0;
+            if (k < nk) {
 #pragma unroll
-            for (int i = 0; i < kQConsumers / 32; ++i) acc += (double)sh.part[k][lane + 32 * i];
-            s[k] = acc;
+                for (int i = 0; i < kQConsumers / 32; ++i) acc += (double)sh.part[k][lane + 32 * i];
+            }
+            rs.s[k] = acc;
         }
-        double zr = 0.0, tr = 0.0;
+        rs.zpart = rs.tr = 0.0;
         if (lane < kQWarps) {
-            zr = (double)sh.info.zt[lane].x;
-            tr = (double)sh.info.zt[lane].y;
+            rs.zpart = (double)sh.info.zt[lane].x;
+            rs.tr = (double)sh.info.zt[lane].y;
         }
         const long long lr = sh.info.lr, pr = sh.info.pr;
-        const float m = sh.info.m;
-        const int argmin = sh.info.argmin;
-        const double zmax = (double)sh.info.nmax * (double)sh.info.e0;  // the maxima, left out of the partial sums
-        const int status = sh.info.status;
-        const RowConst rc = sh.info.rc;
-        named_bar_arrive(kBarFree, kQBlock);  // the consumers may refill the buffer from here on
+        const float m = sh.info.m, e0 = sh.info.e0, c0 = sh.info.c0, th = sh.info.th;
+        const int argmin = sh.info.argmin, nmax = sh.info.nmax;
+        int nlist = sh.nlist;
+        nlist = nlist > kListCap ? kListCap : nlist;
+        const bool series = !status && rc.series;
+        double ex = 0.0;
+        float e_first = 0.f;  // this lane's listed code among the first 32
+        if (series) {
+            if (lane < nlist) e_first = sh.list[lane];
+            for (int i = lane; i < nlist; i += 32) ex += (double)sh.list[i] - (double)th;
+        }
+        rs.excess = ex;
+        // Up to 32 listed codes travel in registers and the buffer goes back to the consumers at
+        // once; a longer list is read in place, so the buffer is held until the row is done.
+        const bool hold = series && nlist > 32;
+        if (!hold) {
+            __syncwarp();
+            if (lane == 0) sh.nlist = 0;
+            named_bar_arrive(kBarFree, kQBlock);
+        }
 #pragma unroll
-        for (int k = 0; k < 5; ++k) s[k] = warp_sum_d(s[k]);
-        zr = warp_sum_d(zr) + zmax;
-        tr = warp_sum_d(tr);
-        if (lane == 0) finalize_one(a, s, zr, tr, lr, pr, m, argmin, status, rc);
+        for (int k = 0; k < 5; ++k) rs.s[k] = warp_sum_d(rs.s[k]);
+        rs.zpart = warp_sum_d(rs.zpart);
+        rs.tr = warp_sum_d(rs.tr);
+        rs.excess = warp_sum_d(rs.excess);
+
+        double S_lo = 0.0, S_up = 0.0, omega = 0.0, sigma = 0.0;
+        if (series) {
+            if (!(rc.rho == beta_key)) {
+                double r = (double)rc.rho;
+                if (a.radius_is_raw) r = (r > 0.0) ? r + log1p(exp(-r)) : log1p(exp(r));  // Softplus, beta = 1
+                if (r > (double)a.r_max) r = (double)a.r_max;
+                beta_val = expm1(r);
+                beta_key = rc.rho;
+            }
+            series_sums(a, sh, rs, beta_val, e0, nmax, c0, th, nlist, e_first, lane, S_lo, S_up, omega, sigma);
+        } else if (!status) {
+            direct_sums(a, rs, rc, S_lo, S_up, omega, sigma);
+        }
+        if (hold) {
+            __syncwarp();
+            if (lane == 0) sh.nlist = 0;
+            named_bar_arrive(kBarFree, kQBlock);
+        }
+        if (lane == 0) {
+            if (status) {
+                write_unusable(o, lr, status);
+            } else {
+                const double score = omega * sigma;
+                // exponent actually used: c * log2e_f - m2 = (c - m) * log2e_f + off with off = m * log2e_f - m2
+                const double off = (double)m * (double)kLog2e - (double)(m * kLog2e);
+                const double unscale = exp2(-off);
+                const double z = (rs.zpart + (double)nmax * (double)e0) * unscale;
+                const double t = rs.tr * unscale - off * z;
+                const double lnz = log(z);
+                const double entropy = lnz - kLn2D * t / z;
+                const double p_max = 1.0 / z;
+                int fl;
+                switch (a.policy) {
+                case CIAR_POLICY_INTERVAL: fl = score > (double)a.tau; break;
+                case CIAR_POLICY_ENTROPY: fl = entropy > (double)a.tau; break;
+                case CIAR_POLICY_MAXPROB: fl = p_max < (double)a.tau; break;
+                case CIAR_POLICY_RANDOM: fl = a.u_flag[pr] < a.tau; break;
+                default: fl = 1; break;
+                }
+                if (o.row_max) o.row_max[lr] = m;
+                if (o.sum_exp) o.sum_exp[lr] = (float)z;
+                if (o.lse) o.lse[lr] = (float)((double)m + lnz);
+                if (o.p_max) o.p_max[lr] = (float)p_max;
+                if (o.entropy) o.entropy[lr] = (float)entropy;
+                if (o.S_lo) o.S_lo[lr] = (float)S_lo;
+                if (o.S_up) o.S_up[lr] = (float)S_up;
+                if (o.omega) o.omega[lr] = (float)omega;
+                if (o.sigma) o.sigma[lr] = (float)sigma;
+                if (o.score) o.score[lr] = (float)score;
+                if (o.argmax) o.argmax[lr] = argmin + a.vb;
+                if (o.flag) o.flag[lr] = (uint8_t)fl;
+                if (o.row_status) o.row_status[lr] = 0;
+            }
+        }
         __syncwarp();
     }
 }
 
 template <typename T, int JV, int MINB>
-__global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(QuantifyArgs a)
+__global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __grid_constant__ QuantifyArgs a)
 {
     constexpr int VEC = Elem<T>::kVec;
     constexpr int NPV = VEC / 2;  // float2 pairs per 16-byte vector
@@ -323,6 +456,7 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(Quantify
 #pragma unroll
         for (int s = 0; s < kQStages; ++s) mbar_init(&sh.full[s], 1);
         sh.abort = 0;
+        sh.nlist = 0;
         sh.info.cmd = 0;
         mbar_init_fence();
     }
@@ -339,6 +473,7 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(Quantify
     const T *base = reinterpret_cast<const T *>(a.logits) + a.vb;
     const ciar_quantify_out &o = a.out;
     const int64_t stride_rows = gridDim.x;
+    const float inv_n = 1.0f / (float)a.n;
 
     // issues the copy of this CTA's k-th row into its stage (thread 0 only)
     auto issue = [&](int k) {
@@ -435,20 +570,17 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(Quantify
             }
         }
         float zs = z2.x + z2.y;
+        const float e0 = ex2_approx(fmaf(m, kLog2e, -m2));  // the exponential every maximum got
         if (tm == m) {
             // This thread owns a maximum.  A term near 1 would cost the small terms their low bits, so its
-            // partial sum is formed again without the maxima; they come back exactly, as a count times e0.
+            // partial sum is formed again without the terms equal to e0; they come back exactly, as a count.
             float zz = 0.f;
             int cnt = 0;
 #pragma unroll
-            for (int j = 0; j < JV; ++j) {
-#pragma unroll
-                for (int q = 0; q < NPV; ++q) {
-                    if (j < nj) {
-                        const float2 c = row.pair(j, q), ev = e[j * NPV + q];
-                        if (c.x == m) ++cnt; else zz += ev.x;
-                        if (c.y == m) ++cnt; else zz += ev.y;
-                    }
+            for (int i = 0; i < NP; ++i) {
+                if (i / NPV < nj) {
+                    if (e[i].x == e0) ++cnt; else zz += e[i].x;
+                    if (e[i].y == e0) ++cnt; else zz += e[i].y;
                 }
             }
             zs = zz;
@@ -460,13 +592,12 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(Quantify
         float z = sh.wz[lane & (kQWarps - 1)];
 #pragma unroll
         for (int ofs = 8; ofs > 0; ofs >>= 1) z += __shfl_xor_sync(0xffffffffu, z, ofs);
-        const float e0 = ex2_approx(fmaf(m, kLog2e, -m2));  // the exponential every maximum got
         const int nmax = sh.nmax;
         z = fmaf((float)nmax, e0, z);
         const RowConst rc = sh.rc[k & 1];
 
         int status = 0;
-        if (!(m > kLogitFloor) || !(z > 0.f) || !(z < INFINITY) || !(rc.r == rc.r)) {
+        if (!(m > kLogitFloor) || !(z > 0.f) || !(z < INFINITY) || !(rc.rho == rc.rho)) {
             // an unusable row (NaN / +inf logit, no finite logit, NaN radius): classify it from the
             // landed bytes exactly as the row-status bits are defined
             if (tid == 0) sh.bad_nan = sh.bad_finite = 0;
@@ -487,57 +618,114 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(Quantify
             if (has_nan) sh.bad_nan = 1;
             if (has_finite) sh.bad_finite = 1;
             named_bar_sync(kBarConsumers, kQConsumers);
-            if (sh.bad_nan || !(rc.r == rc.r)) status |= CIAR_ROW_NAN;
+            if (sh.bad_nan || !(rc.rho == rc.rho)) status |= CIAR_ROW_NAN;
             if (!sh.bad_finite) status |= CIAR_ROW_NO_FINITE;
             if (!status) status = CIAR_ROW_NAN;  // sums overflowed without any single bad logit
         }
-        if (tid == 0) {  // every consumer has read the stage: refill it
+        const bool direct = !status && !rc.series;
+        if (tid == 0 && !direct) {  // every consumer has read the stage: refill it
             fence_proxy_async_smem();
             issue(k + kQStages);
         }
+        // the hand-off buffer (partial sums, list of large codes) must be free from here on
+        named_bar_sync(kBarFree, kQBlock);
 
-        // ---- sweep 3: interval sums from the exponentials in registers
-        float2 P1 = f2(0.f), D1 = f2(0.f), PP = f2(0.f), PD = f2(0.f), DD = f2(0.f);
-        if (!status) {
-            const float invz = 1.0f / z;
-            const float2 iz = f2(invz), niz = f2(-invz), one = f2(1.0f);
-            const float2 a1 = f2(rc.a1), b1 = f2(rc.b1), npl0 = f2(-rc.pl0), ndd0 = f2(-rc.dd0);
+        // ---- sweep 3: interval sums
+        float ps[5] = { 0.f, 0.f, 0.f, 0.f, 0.f };
+        const float c0 = z * inv_n, th = rc.theta_p * z;
+        if (!status && rc.series) {
+            // power sums of (e - c0) from the exponentials in registers; codes above th are clamped and listed
+            float2 T2 = f2(0.f), T3 = f2(0.f), T4 = f2(0.f);
+            const float2 nc0 = f2(-c0);
+            const float e_tm = ex2_approx(fmaf(tm, kLog2e, -m2));  // this thread's largest exponential
+            if (!__any_sync(0xffffffffu, e_tm > th)) {
 #pragma unroll
-            for (int i = 0; i < NP; ++i) {
-                if (i / NPV < nj) {
-                    const float2 x = __fmul2_rn(e[i], iz);
-                    const float2 sx = __ffma2_rn(e[i], niz, one);
-                    const float2 den_l = __ffma2_rn(b1, sx, a1);
-                    const float2 den_u = __ffma2_rn(b1, x, a1);
-                    const float2 q = __fmul2_rn(den_l, den_u);
-                    const float2 xr = __fmul2_rn(x, make_float2(rcp_approx(q.x), rcp_approx(q.y)));
-                    const float2 pl = __ffma2_rn(__fmul2_rn(xr, den_u), a1, npl0);  // p^l term minus its centre
-                    const float2 dd = __ffma2_rn(xr, sx, ndd0);                     // width term minus its centre
-                    P1 = __fadd2_rn(P1, pl);
-                    D1 = __fadd2_rn(D1, dd);
-                    PP = __ffma2_rn(pl, pl, PP);
-                    PD = __ffma2_rn(pl, dd, PD);
-                    DD = __ffma2_rn(dd, dd, DD);
+                for (int i = 0; i < NP; ++i) {
+                    if (i / NPV < nj) {
+                        const float2 y = __fadd2_rn(e[i], nc0);
+                        const float2 y2 = __fmul2_rn(y, y);
+                        T2 = __fadd2_rn(T2, y2);
+                        T3 = __ffma2_rn(y2, y, T3);
+                        T4 = __ffma2_rn(y2, y2, T4);
+                    }
                 }
+            } else {
+#pragma unroll
+                for (int i = 0; i < NP; ++i) {
+                    if (i / NPV < nj) {
+                        float2 ev = e[i];
+                        if (ev.x > th) {
+                            const int slot = atomicAdd(&sh.nlist, 1);
+                            if (slot < kListCap) sh.list[slot] = ev.x;
+                            ev.x = th;
+                        }
+                        if (ev.y > th) {
+                            const int slot = atomicAdd(&sh.nlist, 1);
+                            if (slot < kListCap) sh.list[slot] = ev.y;
+                            ev.y = th;
+                        }
+                        const float2 y = __fadd2_rn(ev, nc0);
+                        const float2 y2 = __fmul2_rn(y, y);
+                        T2 = __fadd2_rn(T2, y2);
+                        T3 = __ffma2_rn(y2, y, T3);
+                        T4 = __ffma2_rn(y2, y2, T4);
+                    }
+                }
+            }
+            ps[0] = T2.x + T2.y;
+            ps[1] = T3.x + T3.y;
+            ps[2] = T4.x + T4.y;
+        } else if (direct) {
+            // both bounds of every code, from the row still sitting in its stage
+            const float invz = 1.0f / z;
+            float P1 = 0.f, D1 = 0.f, PP = 0.f, PD = 0.f, DD = 0.f;
+#pragma unroll 1
+            for (int j = 0; j < nj; ++j) {
+                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQConsumers) * 16);
+                float c[VEC];
+                Elem<T>::load(v, c);
+#pragma unroll
+                for (int q = 0; q < VEC; ++q) {
+                    const float ev = ex2_approx(fmaf(c[q], kLog2e, -m2));
+                    const float x = ev * invz, sx = fmaf(-ev, invz, 1.0f);
+                    const float den_l = fmaf(rc.b1, sx, rc.a1), den_u = fmaf(rc.b1, x, rc.a1);
+                    const float xr = x * rcp_approx(den_l * den_u);
+                    const float pl = fmaf(xr * den_u, rc.a1, -rc.pl0);  // p^l term minus its centre
+                    const float dd = fmaf(xr, sx, -rc.dd0);             // width term minus its centre
+                    P1 += pl;
+                    D1 += dd;
+                    PP = fmaf(pl, pl, PP);
+                    PD = fmaf(pl, dd, PD);
+                    DD = fmaf(dd, dd, DD);
+                }
+            }
+            ps[0] = P1; ps[1] = D1; ps[2] = PP; ps[3] = PD; ps[4] = DD;
+            named_bar_sync(kBarConsumers, kQConsumers);
+            if (tid == 0) {
+                fence_proxy_async_smem();
+                issue(k + kQStages);
             }
         }
 
         // ---- hand the row to the finalizer warp
-        named_bar_sync(kBarFree, kQBlock);
-        sh.part[0][tid] = P1.x + P1.y;
-        sh.part[1][tid] = D1.x + D1.y;
-        sh.part[2][tid] = PP.x + PP.y;
-        sh.part[3][tid] = PD.x + PD.y;
-        sh.part[4][tid] = DD.x + DD.y;
+        sh.part[0][tid] = ps[0];
+        sh.part[1][tid] = ps[1];
+        sh.part[2][tid] = ps[2];
+        if (direct) {
+            sh.part[3][tid] = ps[3];
+            sh.part[4][tid] = ps[4];
+        }
         if (lane == 0) sh.info.zt[warp].x = zt;
         if (lane == 16) sh.info.zt[warp].y = zt;
         if (tid == 0) {
             sh.info.lr = lr;
             sh.info.pr = pr;
             sh.info.m = m;
+            sh.info.e0 = e0;
+            sh.info.c0 = c0;
+            sh.info.th = th;
             sh.info.argmin = sh.argmin;
             sh.info.nmax = nmax;
-            sh.info.e0 = e0;
             sh.info.status = status;
         }
         if (tid == 32) sh.info.rc = rc;
