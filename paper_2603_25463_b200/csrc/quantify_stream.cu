@@ -1,13 +1,13 @@
 // Streaming quantifier for rows that fit on chip (2048 .. 16384 codes, scalar or per-row radius).
 //
-// One persistent CTA walks rows blockIdx.x, blockIdx.x + gridDim.x, ...  Rows arrive through a
-// ring of shared-memory stages filled by bulk (TMA) copies that one thread issues several rows
-// ahead, so HBM always has requests in flight.  16 consumer warps sweep a landed row twice from
-// shared memory (maximum; then one exponential per code, kept in registers: 32 per thread) and
-// once more from those registers (interval sums).  A 17th warp, fed through a small hand-off
-// buffer, reduces the per-thread sums, works out the interval constants of the rows to come,
-// and does the per-row double-precision arithmetic for 16 rows at a time, one row per lane, off
-// the consumers' critical path.  Each logit is read from HBM once.
+// One persistent CTA of 16 warps walks rows blockIdx.x, blockIdx.x + gridDim.x, ...  Rows arrive
+// through a ring of shared-memory stages filled by bulk (TMA) copies that one thread issues
+// several rows ahead, so HBM always has requests in flight.  The warps sweep a landed row twice
+// from shared memory (maximum; then one exponential per code, kept in registers: 32 per thread)
+// and once more from those registers (interval sums), reduce their sums with shuffles and park
+// them in shared memory.  Every 16 rows the CTA stops for a moment and each warp finishes one
+// parked row: the handful of large codes exactly, one per lane, then the row's double-precision
+// scalar arithmetic and its stores.  Each logit is read from HBM once.
 #include <climits>
 
 #include "ciar_internal.h"
@@ -17,62 +17,44 @@ namespace ciar {
 
 namespace {
 
-constexpr int kQConsumers = 512;
-constexpr int kQWarps = kQConsumers / 32;
-constexpr int kQBlock = kQConsumers + 32;  // + the finalizer warp
+constexpr int kQThreads = 512;
+constexpr int kQWarps = kQThreads / 32;
 constexpr int kQStages = 3;
-constexpr int kBarConsumers = 1, kBarFull = 2, kBarFree = 3;  // named barriers
-constexpr long long kWaitCycles = 2000000000ll;                // bound of a wait for a row (about a second)
-constexpr long long kDrainCycles = 20000000ll;                 // bound of each wait while leaving after a failure
-// Logits at or below -2^120 are treated as -inf (their exponential is 0 either way); the floor
-// keeps 0 * (-inf) out of the entropy sum.
-constexpr float kLogitFloor = -1.329227995784916e36f;
-constexpr uint32_t kLogitFloorBf16x2 = 0xFB80FB80u;
+constexpr int kBarRow = 1;                       // named barrier of the row sweeps
+constexpr long long kWaitCycles = 2000000000ll;  // bound of a wait for a row (about a second)
+constexpr long long kDrainCycles = 20000000ll;   // bound of each wait while leaving after a failure
 
-// Interval constants of one row.
-//
-// With x = softmax probability, s = 1 - x and beta = e^r - 1 the raw InterFuse bounds are
+// The interval arithmetic.  With x = softmax probability, s = 1 - x and beta = e^r - 1 the raw
+// InterFuse bounds are
 //   p^l = x / (1 + beta s),   p^u = (1 + beta) x / (1 + beta x),
 //   p^u - p^l = beta (2 + beta) x s / ((1 + beta s)(1 + beta x)).
-// Rows with r <= 1 take the "series" route: every code with x below theta = 2^-8 / (1 + beta) enters
-// only through the power sums of (e - c0) up to the fourth (c0 = Z / n), from which the finalizer
-// rebuilds the sums of p^l, of the widths and of their squares by a fourth-order Taylor expansion
-// about x0 = 1 / n (terms beyond it are below 1e-7 of the result); the few codes above theta are
-// clamped to it in the power sums, listed, and put back exactly.  Rows with r > 1 take the
-// "direct" route: both bounds of every code from the formulas above, in the scaled form
-//   den_l = a1 + b1 s, den_u = a1 + b1 x, (a1, b1) = (1, beta) or (1 / beta, 1) for beta > 1,
-// which keeps every term in range for radii up to 80.
-struct RowConst {
-    float rho;       // radius as stored (before Softplus when raw); NaN marks an unusable radius
-    float theta_p;   // series route: probability above which a code is treated exactly
-    float a1, b1;    // direct route
-    float pl0, dd0;  // direct route: the two raw terms at x = 1 / n, about which its sums are taken
-    int series;
+// Rows with r <= 1 take the "series" route: every code with x below theta = 2^-8 e^-r enters only
+// through the power sums of (e - c0) up to the fourth (e = exp(c - m), c0 = Z / n), from which the
+// sums of p^l, of the widths and of their squares are rebuilt by a fourth-order Taylor expansion
+// about x0 = 1 / n (terms beyond it are below 1e-7 of the result); the few codes above theta
+// (fewer than 256 e^r) are clamped to it in the power sums, listed, and put back exactly.  Rows
+// with r > 1 take the "direct" route: both bounds of every code from the formulas above, in the
+// scaled form den_l = a1 + b1 s, den_u = a1 + b1 x with (a1, b1) = (1, beta) or (1 / beta, 1) for
+// beta > 1, which keeps every term in range for radii up to 80.
+struct DirectConst {
+    float a1, b1;
+    float pl0, dd0;  // the two raw terms at x = 1 / n, about which the direct sums are taken
     int big;
 };
 
-constexpr int kListCap = 704;  // > 256 (1 + beta) for r <= 1: more codes than that cannot exceed theta
-constexpr int kBatch = 16;     // rows finalized together, one per lane (of the first 16)
+constexpr int kPark = 16;      // rows parked before the CTA finishes them, one per warp
+constexpr int kListCap = 704;  // > 256 e for r <= 1: more codes than that cannot exceed theta
+constexpr int kParkList = 48;  // listed codes a parked row can carry; a longer list is finished at once
 
-// What the consumers hand over with one row.
-struct RowInfo {
+// A row whose sweeps are done and whose arithmetic is still to do.
+struct Parked {
+    float wsum[kQWarps][7];  // per-warp sums: 0 exp (terms equal to e0 left out), 1 exp * exponent, 2.. route sums
+    float list[kParkList];   // series route: exponentials of the codes above theta
     long long lr, pr;
-    float m, e0;   // row maximum; the exponential of a code equal to it, as the consumers computed it
+    float m, e0;   // row maximum; the exponential of a code equal to it, as the sweeps computed it
     float c0, th;  // series route: centre of the power sums and clamp level, in units of exp(c - m)
-    int argmin, nmax;
-    int status;  // CIAR_ROW_* bits found by the consumers (0 = a regular row)
-    int cmd;     // 0 = finalize this row, 1 = no more rows, 2 = a skipped row (nothing to finalize)
-    float2 zt[kQWarps];  // per-warp sums of exp (terms equal to e0 left out) and of exp * exponent
-};
-
-// Rows whose sums are complete and that wait for their scalar arithmetic (struct of arrays, one slot per lane).
-struct Batch {
-    double v[11][kBatch];  // series: power sums 2..4, zpart, tr, excess, five sums over listed codes; direct: five sums, zpart, tr
-    double beta[kBatch];
-    long long lr[kBatch], pr[kBatch];
-    float m[kBatch], e0[kBatch], c0[kBatch], th[kBatch];
-    int argmin[kBatch], nmax[kBatch], nlist[kBatch], status[kBatch];
-    RowConst rc[kBatch];
+    float rho, r;  // radius as stored, and clamped (after Softplus when raw) as the sweeps used it
+    int argmin, nmax, nlist, status, series;
 };
 
 struct QShared {
@@ -82,29 +64,24 @@ struct QShared {
     int argmin, nmax;  // lowest index holding the row maximum, number of codes whose exponential equals e0
     int bad_nan, bad_finite;
     int abort;
-    int nlist;  // codes above theta in the row being swept (reset by the finalizer when it has read them)
-    RowInfo info;
-    RowConst rc_tab[2][kBatch];  // interval constants of this CTA's rows kBatch b .. kBatch (b + 1) - 1 in rc_tab[b & 1]
-    double beta_tab[2][kBatch];  // e^r - 1 of the same rows, in double
-    float part[3][kQConsumers];  // series route: per-thread power sums
-    float dpart[5][kQWarps];     // direct route: per-warp sums
+    int nlist;  // codes above theta in the row being swept
     float list[kListCap];
-    Batch batch;
+    Parked park[kPark];
 };
 static_assert(sizeof(QShared) + kQStages * 32768 <= 115712, "two CTAs per SM must fit in shared memory");
 
-// Interval constants of a row from its stored radius (float for the consumers, beta in double for the finalizer).
-__device__ __forceinline__ RowConst make_row_const(float rho, int raw, float r_max, int n, double &beta_d)
+// Clamped radius of a row from its stored value (Softplus when raw), in float for the sweeps.
+__device__ __forceinline__ float row_radius(float rho, int raw, float r_max)
 {
-    RowConst k;
-    k.rho = rho;
-    double rd = (double)rho;
-    if (raw) rd = (rd > 0.0) ? rd + log1p(exp(-rd)) : log1p(exp(rd));  // Softplus, beta = 1
-    if (rd > (double)r_max) rd = (double)r_max;
-    beta_d = expm1(rd);
-    const float r = (float)rd, beta = (float)beta_d;
-    k.series = r <= 1.0f;
-    k.theta_p = 0.00390625f / (1.0f + beta);
+    float r = rho;
+    if (raw) r = (rho > 0.f) ? rho + log1pf(expf(-rho)) : log1pf(expf(rho));  // Softplus, beta = 1
+    return fminf(r, r_max);
+}
+
+__device__ __forceinline__ DirectConst make_direct_const(float r, int n)
+{
+    DirectConst k;
+    const float beta = expm1f(r);
     k.big = beta > 1.0f;
     if (k.big) {
         k.a1 = 1.0f / beta;
@@ -122,8 +99,7 @@ __device__ __forceinline__ RowConst make_row_const(float rho, int raw, float r_m
 }
 
 // A 16-byte vector of a landed row.  fold_max() folds it into a running maximum (bf16: two packed
-// halves), pairs() widens it to float2 pairs with -inf floored (a NaN stays a NaN), find() gives the
-// position of the first code equal to m.
+// halves, NaN ignored), pairs() widens it to float2 pairs.
 template <typename T>
 struct Vec;
 
@@ -131,7 +107,7 @@ template <>
 struct Vec<__nv_bfloat16> {
     static constexpr int kPairs = 4;
     typedef uint32_t Max;
-    static __device__ __forceinline__ Max max_init() { return kLogitFloorBf16x2; }
+    static __device__ __forceinline__ Max max_init() { return 0xFF80FF80u; }  // (-inf, -inf)
     static __device__ __forceinline__ Max fold_max(Max mx, const uint4 &v)
     {
         return bf16x2_max(mx, bf16x2_max(bf16x2_max(v.x, v.y), bf16x2_max(v.z, v.w)));
@@ -143,14 +119,11 @@ struct Vec<__nv_bfloat16> {
     }
     static __device__ __forceinline__ void pairs(const uint4 &v, float2 (&c)[4])
     {
-        uint32_t w[4] = { v.x, v.y, v.z, v.w };
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            asm("max.NaN.bf16x2 %0, %0, %1;" : "+r"(w[q]) : "r"(kLogitFloorBf16x2));
-            c[q] = unpack_bf16x2(w[q]);
-        }
+        c[0] = unpack_bf16x2(v.x);
+        c[1] = unpack_bf16x2(v.y);
+        c[2] = unpack_bf16x2(v.z);
+        c[3] = unpack_bf16x2(v.w);
     }
-    static __device__ __forceinline__ float2 exponent_for_entropy(float2 d) { return d; }  // floored already
 };
 
 template <>
@@ -169,16 +142,19 @@ struct Vec<float> {
         c[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
         c[1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
     }
-    // -inf logit: exp = 0 and the exponent is floored so that the product is 0, not NaN
-    static __device__ __forceinline__ float2 exponent_for_entropy(float2 d)
-    {
-        return make_float2(fmaxf(d.x, kNegHuge), fmaxf(d.y, kNegHuge));
-    }
 };
 
 __device__ __forceinline__ const uint4 &stage_vec(const unsigned char *stage, int vi)
 {
     return *reinterpret_cast<const uint4 *>(stage + (size_t)vi * 16);
+}
+
+// 1 / x for a positive normal double: a float reciprocal refined by two Newton steps (full double accuracy)
+__device__ __forceinline__ double fast_rcp(double x)
+{
+    double r = (double)rcp_approx((float)x);
+    r = fma(r, fma(-x, r, 1.0), r);
+    return fma(r, fma(-x, r, 1.0), r);
 }
 
 __device__ __forceinline__ double warp_sum_d(double v)
@@ -207,80 +183,104 @@ __device__ __forceinline__ void write_unusable(const ciar_quantify_out &o, long 
     if (o.row_status) o.row_status[lr] = (uint8_t)status;
 }
 
-// Slots of Batch::v.  Both routes: 0 zpart (sum of exponentials without the terms equal to e0), 1 the
-// entropy sum.  Series route: 2..4 power sums of (e - c0), 5 sum over listed codes of (e - clamp),
-// 6..10 sums over listed codes of p^l, d, p^l^2, p^l d, d^2 (exact, d = p^u - p^l).  Direct route:
-// 2..6 the five centred sums.
-enum { kVZ = 0, kVT = 1, kVS = 2, kVEx = 5, kVL = 6 };
 
-// Scalar arithmetic of one finished row (normalisation step, Omega, Sigma, U, entropy, the flag)
-// and its stores.  Called with one row per lane.
-__device__ __forceinline__ void finalize_slot(const QuantifyArgs &a, const Batch &bt, int slot)
+// Finishes one row whose sums are parked: reduces the per-warp sums, treats the listed codes
+// exactly (one per lane), then does the scalar arithmetic (normalisation step, Omega, Sigma, U,
+// entropy, the flag) and the stores.  Run by one whole warp.
+__device__ __noinline__ void finish_row(const QuantifyArgs &a, const Parked &pk, const float *list, int lane)
 {
     const ciar_quantify_out &o = a.out;
-    const long long lr = bt.lr[slot], pr = bt.pr[slot];
-    const int status = bt.status[slot];
-    if (status) {
-        write_unusable(o, lr, status);
+    const long long lr = pk.lr;
+    if (pk.status) {
+        if (lane == 0 && pk.status > 0) write_unusable(o, lr, pk.status);  // negative: finished earlier
         return;
     }
-    const RowConst rc = bt.rc[slot];
-    const double nn = (double)a.n;
-    const double e0 = (double)bt.e0[slot];
-    const int nmax = bt.nmax[slot];
-    const double zd = bt.v[kVZ][slot] + (double)nmax * e0;  // the row's sum of exponentials
+    const bool series = pk.series != 0;
+    double v[7];
+#pragma unroll
+    for (int q = 0; q < 7; ++q) {
+        v[q] = 0.0;
+        if (q < 5 || !series) {
+            if (lane < kQWarps) v[q] = (double)pk.wsum[lane][q];
+            v[q] = warp_sum_d(v[q]);
+        }
+    }
+    const double nn = (double)a.n, inv_nn = fast_rcp(nn);
+    const double e0 = (double)pk.e0;
+    const int nmax = pk.nmax;
+    const double zpart = v[0], zd = zpart + (double)nmax * e0;  // the row's sum of exponentials
+    const double beta = (double)expm1f(pk.r);  // e^r - 1 to float accuracy: the bounds depend on it smoothly
     double S_lo, S_up, omega, ss;
-    if (rc.series) {
-        const double beta = bt.beta[slot];
-        const double nl = (double)bt.nlist[slot];
-        const double c0 = (double)bt.c0[slot], th = (double)bt.th[slot];
-        const double invz = 1.0 / zd;
+    if (series) {
+        const int nlist = pk.nlist < kListCap ? pk.nlist : kListCap;
+        const double c0 = (double)pk.c0, th = (double)pk.th;
+        const double invz = fast_rcp(zd);
         const double b = 1.0 + beta, kap = beta * (2.0 + beta);
+        // listed codes, exactly: sums of e - clamp, p^l, d, p^l^2, p^l d, d^2 (d = p^u - p^l)
+        double ls[6] = { 0.0, 0.0, 0.0, 0.0, 0.0, 0.0 };
+        for (int i = lane; i < nlist; i += 32) {
+            const double e = (double)list[i];
+            const double x = e * invz;
+            // 1 - x from the other codes' exponentials (no cancellation for a dominant code)
+            const double sx = (e == e0 ? zpart + (double)(nmax - 1) * e0 : zd - e) * invz;
+            const double den = fast_rcp((1.0 + beta * sx) * (1.0 + beta * x));
+            const double pl = x * (1.0 + beta * x) * den, d = kap * x * sx * den;
+            ls[0] += e - th;
+            ls[1] += pl;
+            ls[2] += d;
+            ls[3] += pl * pl;
+            ls[4] += pl * d;
+            ls[5] += d * d;
+        }
+        if (nlist > 0) {
+#pragma unroll
+            for (int q = 0; q < 6; ++q) ls[q] = warp_sum_d(ls[q]);
+        }
+        const double nl = (double)nlist;
         const double x0 = c0 * invz, hth = (th - c0) * invz;
         const double iz2 = invz * invz;
-        const double H1 = (zd - bt.v[kVEx][slot] - nn * c0) * invz;  // sum of (clamped x - x0)
-        const double H2 = bt.v[kVS][slot] * iz2, H3 = bt.v[kVS + 1][slot] * iz2 * invz, H4 = bt.v[kVS + 2][slot] * iz2 * iz2;
+        const double H1 = (zd - ls[0] - nn * c0) * invz;  // sum of (clamped x - x0)
+        const double H2 = v[2] * iz2, H3 = v[3] * iz2 * invz, H4 = v[4] * iz2 * iz2;
         // Taylor coefficients about x0 of p^l(x) = x / (b - beta x) and p^u(x) = b x / (1 + beta x)
-        const double u = b - beta * x0, v = 1.0 + beta * x0;
-        const double iuv = 1.0 / (u * v), iu = v * iuv, iv = u * iuv;
-        const double rl = beta * iu, ru = -beta * iv;
+        const double u = b - beta * x0, w = 1.0 + beta * x0;
+        const double iuw = fast_rcp(u * w), iu = w * iuw, iw = u * iuw;
+        const double rl = beta * iu, ru = -beta * iw;
         const double PL0 = x0 * iu, PL1 = b * iu * iu, PL2 = PL1 * rl, PL3 = PL2 * rl, PL4 = PL3 * rl;
-        const double PU1 = b * iv * iv, PU2 = PU1 * ru, PU3 = PU2 * ru, PU4 = PU3 * ru;
-        const double DD0 = kap * x0 * (1.0 - x0) * iuv;                        // p^u - p^l at x0, no cancellation
-        const double DD1 = b * beta * (1.0 - 2.0 * x0) * (u + v) * iuv * iuv;  // PU1 - PL1, no cancellation
+        const double PU1 = b * iw * iw, PU2 = PU1 * ru, PU3 = PU2 * ru, PU4 = PU3 * ru;
+        const double DD0 = kap * x0 * (1.0 - x0) * iuw;                        // p^u - p^l at x0, no cancellation
+        const double DD1 = b * beta * (1.0 - 2.0 * x0) * (u + w) * iuw * iuw;  // PU1 - PL1, no cancellation
         const double DD2 = PU2 - PL2, DD3 = PU3 - PL3, DD4 = PU4 - PL4;
         const double h2 = hth * hth, h3 = h2 * hth, h4 = h2 * h2;
         // what a code clamped to theta contributed through the power sums
         const double pl_th = PL0 + PL1 * hth + PL2 * h2 + PL3 * h3 + PL4 * h4;
         const double dd_th = DD0 + DD1 * hth + DD2 * h2 + DD3 * h3 + DD4 * h4;
-        const double lpl = bt.v[kVL][slot], ld = bt.v[kVL + 1][slot], lpp = bt.v[kVL + 2][slot],
-                     lpd = bt.v[kVL + 3][slot], ldd = bt.v[kVL + 4][slot];
-        const double B = nn * PL0 + PL1 * H1 + PL2 * H2 + PL3 * H3 + PL4 * H4 + (lpl - nl * pl_th);  // sum of raw p^l
-        const double A = nn * DD0 + DD1 * H1 + DD2 * H2 + DD3 * H3 + DD4 * H4 + (ld - nl * dd_th);   // sum of raw widths
+        const double B = nn * PL0 + PL1 * H1 + PL2 * H2 + PL3 * H3 + PL4 * H4 + (ls[1] - nl * pl_th);  // sum of raw p^l
+        const double A = nn * DD0 + DD1 * H1 + DD2 * H2 + DD3 * H3 + DD4 * H4 + (ls[2] - nl * dd_th);  // sum of raw widths
         S_lo = B;
         S_up = A + B;
-        const double rs = 1.0 / (S_lo * S_up);
+        const double rs = S_lo > 0.0 && S_up > 0.0 ? fast_rcp(S_lo * S_up) : 0.0;
         double k_lo = (double)a.lo_cap * S_up * rs, k_up = (double)a.hi_cap * S_lo * rs;
         if (!(S_lo > 0.0) || !(k_lo < 1.0)) k_lo = 1.0;
         if (!(S_up > 0.0) || !(k_up > 1.0)) k_up = 1.0;
         const double g = k_up - k_lo;  // delta = k_up (p^u - p^l) + g p^l
         omega = k_up * A + g * B;
-        const double mu = omega / nn;
+        const double mu = omega * inv_nn;
         const double E0 = k_up * DD0 + g * PL0 - mu, E1 = k_up * DD1 + g * PL1, E2 = k_up * DD2 + g * PL2,
                      E3 = k_up * DD3 + g * PL3, E4 = k_up * DD4 + g * PL4;
         const double q11 = E1 * E1, q12 = 2.0 * E1 * E2, q22 = 2.0 * E1 * E3 + E2 * E2;
         const double sq_th = E0 * E0 + 2.0 * E0 * (E1 * hth + E2 * h2 + E3 * h3 + E4 * h4) + q11 * h2 + q12 * h3 + q22 * h4;
         // listed codes: sum of (delta - mu)^2 from their five exact sums
-        const double sl = k_up * k_up * ldd + 2.0 * k_up * g * lpd + g * g * lpp - 2.0 * mu * (k_up * ld + g * lpl) + nl * mu * mu;
+        const double sl = k_up * k_up * ls[5] + 2.0 * k_up * g * ls[4] + g * g * ls[3] - 2.0 * mu * (k_up * ls[2] + g * ls[1]) +
+                          nl * mu * mu;
         ss = nn * E0 * E0 + 2.0 * E0 * (E1 * H1 + E2 * H2 + E3 * H3 + E4 * H4) + q11 * H2 + q12 * H3 + q22 * H4 +
              (sl - nl * sq_th);
     } else {
-        const double P1 = bt.v[kVS][slot], D1 = bt.v[kVS + 1][slot], PP = bt.v[kVS + 2][slot], PD = bt.v[kVS + 3][slot],
-                     DD = bt.v[kVS + 4][slot];
-        const double a1 = (double)rc.a1, b1 = (double)rc.b1;
-        const double kd = rc.big ? 1.0 + 2.0 * a1 : b1 * (2.0 + b1);
-        const double B = nn * (double)rc.pl0 + P1;  // sum of the raw lower bounds
-        const double Dsum = nn * (double)rc.dd0 + D1;
+        const DirectConst dc = make_direct_const(pk.r, a.n);  // the same constants as the sweep used
+        const double P1 = v[2], D1 = v[3], PP = v[4], PD = v[5], DD = v[6];
+        const double a1 = (double)dc.a1, b1 = (double)dc.b1;
+        const double kd = dc.big ? 1.0 + 2.0 * a1 : b1 * (2.0 + b1);
+        const double B = nn * (double)dc.pl0 + P1;  // sum of the raw lower bounds
+        const double Dsum = nn * (double)dc.dd0 + D1;
         const double A = kd * Dsum;  // sum of the raw widths
         S_lo = B;
         S_up = A + B;
@@ -291,25 +291,28 @@ __device__ __forceinline__ void finalize_slot(const QuantifyArgs &a, const Batch
         const double c1 = k_up * kd, c2 = k_up - k_lo;
         omega = c1 * Dsum + c2 * B;
         const double lin = c1 * D1 + c2 * P1;
-        ss = c1 * c1 * DD + 2.0 * c1 * c2 * PD + c2 * c2 * PP - lin * lin / nn;
+        ss = c1 * c1 * DD + 2.0 * c1 * c2 * PD + c2 * c2 * PP - lin * lin * inv_nn;
     }
-    const double sigma = sqrt((ss > 0.0 ? ss : 0.0) / nn);
+    if (lane != 0) return;
+    const double sigma = sqrt((ss > 0.0 ? ss : 0.0) * inv_nn);
     const double score = omega * sigma;
     // exponent actually used: c * log2e_f - m2 = (c - m) * log2e_f + off with off = m * log2e_f - m2
-    const float m = bt.m[slot];
+    const float m = pk.m;
     const double off = (double)m * (double)kLog2e - (double)(m * kLog2e);
-    const double unscale = exp2(-off);
+    const double w2 = -off * kLn2D;
+    const double unscale = 1.0 + w2 * (1.0 + 0.5 * w2);  // 2^-off: |off| is a rounding error of m * log2e, far below 1e-4
     const double z = zd * unscale;
-    const double t = bt.v[kVT][slot] * unscale - off * z;
-    const double lnz = log(z);
-    const double p_max = 1.0 / z;
+    const double t = v[1] * unscale - off * z;
+    // ln z: z >= 1 up to rounding; log1p keeps the digits of a z just above 1 (a peaked row)
+    const double lnz = z < 1.5 ? (double)log1pf((float)(z - 1.0)) : (double)logf((float)z);
+    const double p_max = fast_rcp(z);
     const double entropy = lnz - kLn2D * t * p_max;
     int fl;
     switch (a.policy) {
     case CIAR_POLICY_INTERVAL: fl = score > (double)a.tau; break;
     case CIAR_POLICY_ENTROPY: fl = entropy > (double)a.tau; break;
     case CIAR_POLICY_MAXPROB: fl = p_max < (double)a.tau; break;
-    case CIAR_POLICY_RANDOM: fl = a.u_flag[pr] < a.tau; break;
+    case CIAR_POLICY_RANDOM: fl = a.u_flag[pk.pr] < a.tau; break;
     default: fl = 1; break;
     }
     if (o.row_max) o.row_max[lr] = m;
@@ -322,163 +325,20 @@ __device__ __forceinline__ void finalize_slot(const QuantifyArgs &a, const Batch
     if (o.omega) o.omega[lr] = (float)omega;
     if (o.sigma) o.sigma[lr] = (float)sigma;
     if (o.score) o.score[lr] = (float)score;
-    if (o.argmax) o.argmax[lr] = bt.argmin[slot] + a.vb;
+    if (o.argmax) o.argmax[lr] = pk.argmin + a.vb;
     if (o.flag) o.flag[lr] = (uint8_t)fl;
     if (o.row_status) o.row_status[lr] = 0;
 }
 
-// Interval constants of this CTA's rows kBatch b .. kBatch b + kBatch - 1, one row per lane of the finalizer warp.
-__device__ __forceinline__ void make_rc_batch(const QuantifyArgs &a, QShared &sh, int b, int lane)
-{
-    const int64_t lr = blockIdx.x + (int64_t)(b * kBatch + lane) * gridDim.x;
-    int64_t pr;
-    float rho = a.r_scalar;
-    if (a.radius_mode == CIAR_RADIUS_PER_ROW) {
-        rho = 0.f;
-        if (lr < a.rows && map_row(a.rm, lr, pr)) rho = reinterpret_cast<const float *>(a.radius)[pr];
-    }
-    double beta;
-    sh.rc_tab[b & 1][lane] = make_row_const(rho, a.radius_is_raw, a.r_max, a.n, beta);
-    sh.beta_tab[b & 1][lane] = beta;
-}
-
-// The finalizer warp.  Per row: take the consumers' partial sums out of the hand-off buffer, give
-// the buffer back, reduce in double, treat the listed codes exactly (one per lane), and park the
-// row in a batch slot.  Per kBatch rows: the scalar arithmetic and the stores, one row per lane.
-__device__ __noinline__ void finalize_rows(const QuantifyArgs &a, QShared &sh, int lane)
-{
-    Batch &bt = sh.batch;
-    if (lane < kBatch) {
-        make_rc_batch(a, sh, 0, lane);
-        make_rc_batch(a, sh, 1, lane);
-    }
-    __syncwarp();
-    named_bar_arrive(kBarFree, kQBlock);
-    int filled = 0;
-    for (int k = 0;; ++k) {
-        named_bar_sync(kBarFull, kQBlock);
-        const int cmd = sh.info.cmd;
-        if (cmd == 1) break;
-        // Every row before k has been handed over, so the table half of the batch before this one
-        // is idle: fill it with the constants of the batch after this one.  The consumers see them
-        // after their next wait on the free barrier.
-        if ((k % kBatch) == 0 && k > 0 && lane < kBatch) make_rc_batch(a, sh, k / kBatch + 1, lane);
-        if (cmd == 2) {  // a row the consumers skipped
-            __syncwarp();
-            named_bar_arrive(kBarFree, kQBlock);
-            continue;
-        }
-        const RowConst rc = sh.rc_tab[(k / kBatch) & 1][k % kBatch];
-        const double beta = sh.beta_tab[(k / kBatch) & 1][k % kBatch];
-        const int status = sh.info.status;
-        const bool series = !status && rc.series;
-        double s[5] = { 0.0, 0.0, 0.0, 0.0, 0.0 };
-        if (series) {
-#pragma unroll
-            for (int q = 0; q < 3; ++q) {
-                double acc = 0.0;
-#pragma unroll
-                for (int i = 0; i < kQConsumers / 32; ++i) acc += (double)sh.part[q][lane + 32 * i];
-                s[q] = acc;
-            }
-        } else if (!status && lane < kQWarps) {
-#pragma unroll
-            for (int q = 0; q < 5; ++q) s[q] = (double)sh.dpart[q][lane];
-        }
-        double zpart = 0.0, tr = 0.0;
-        if (lane < kQWarps) {
-            zpart = (double)sh.info.zt[lane].x;
-            tr = (double)sh.info.zt[lane].y;
-        }
-        const float e0 = sh.info.e0, th = sh.info.th;
-        const int nmax = sh.info.nmax;
-        int nlist = series ? sh.nlist : 0;
-        nlist = nlist > kListCap ? kListCap : nlist;
-        if (lane == 0) {
-            bt.lr[filled] = sh.info.lr;
-            bt.pr[filled] = sh.info.pr;
-            bt.m[filled] = sh.info.m;
-            bt.e0[filled] = e0;
-            bt.c0[filled] = sh.info.c0;
-            bt.th[filled] = th;
-            bt.argmin[filled] = sh.info.argmin;
-            bt.nmax[filled] = nmax;
-            bt.nlist[filled] = nlist;
-            bt.status[filled] = status;
-            bt.rc[filled] = rc;
-            bt.beta[filled] = beta;
-        }
-        const float e_first = lane < nlist ? sh.list[lane] : 0.f;  // this lane's listed code among the first 32
-        // Up to 32 listed codes travel in registers and the buffer goes back to the consumers at
-        // once; a longer list is read in place, so the buffer is held until it has been read.
-        const bool hold = nlist > 32;
-        if (!hold) {
-            __syncwarp();
-            if (lane == 0) sh.nlist = 0;
-            named_bar_arrive(kBarFree, kQBlock);
-        }
-        zpart = warp_sum_d(zpart);
-        tr = warp_sum_d(tr);
-        const int ns = series ? 3 : 5;
-#pragma unroll
-        for (int q = 0; q < 5; ++q)
-            if (q < ns) s[q] = warp_sum_d(s[q]);
-        double ls[6] = { 0.0, 0.0, 0.0, 0.0, 0.0, 0.0 };  // over listed codes: e - clamp, p^l, d, p^l^2, p^l d, d^2
-        if (nlist > 0) {
-            const double e0d = (double)e0, zd = zpart + (double)nmax * e0d, invz = 1.0 / zd;
-            const double kap = beta * (2.0 + beta);
-            for (int i = lane; i < nlist; i += 32) {
-                const double e = i < 32 ? (double)e_first : (double)sh.list[i];
-                const double x = e * invz;
-                // 1 - x from the other codes' exponentials (no cancellation for a dominant code)
-                const double sx = (e == e0d ? zpart + (double)(nmax - 1) * e0d : zd - e) * invz;
-                const double den = 1.0 / ((1.0 + beta * sx) * (1.0 + beta * x));
-                const double pl = x * (1.0 + beta * x) * den, d = kap * x * sx * den;
-                ls[0] += e - (double)th;
-                ls[1] += pl;
-                ls[2] += d;
-                ls[3] += pl * pl;
-                ls[4] += pl * d;
-                ls[5] += d * d;
-            }
-            if (hold) {
-                __syncwarp();
-                if (lane == 0) sh.nlist = 0;
-                named_bar_arrive(kBarFree, kQBlock);
-            }
-#pragma unroll
-            for (int q = 0; q < 6; ++q) ls[q] = warp_sum_d(ls[q]);
-        }
-        if (lane == 0) {
-            bt.v[kVZ][filled] = zpart;
-            bt.v[kVT][filled] = tr;
-#pragma unroll
-            for (int q = 0; q < 5; ++q) bt.v[kVS + q][filled] = s[q];
-            if (series) {
-                bt.v[kVEx][filled] = ls[0];
-#pragma unroll
-                for (int q = 0; q < 5; ++q) bt.v[kVL + q][filled] = ls[1 + q];
-            }
-        }
-        __syncwarp();
-        if (++filled == kBatch) {
-            if (lane < kBatch) finalize_slot(a, bt, lane);
-            filled = 0;
-            __syncwarp();
-        }
-    }
-    if (lane < filled) finalize_slot(a, bt, lane);
-}
-
-// FULL: every consumer thread owns exactly JV vectors (the row has 512 * JV of them).
+// FULL: every thread owns exactly JV vectors (the row has 512 * JV of them).
 template <typename T, int JV, int MINB, bool FULL>
-__global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __grid_constant__ QuantifyArgs a)
+__global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const __grid_constant__ QuantifyArgs a)
 {
     typedef Vec<T> V;
     constexpr int VEC = Elem<T>::kVec;
     constexpr int NPV = V::kPairs;  // float2 pairs per 16-byte vector
     constexpr int NP = JV * NPV;    // pairs per thread
-    constexpr int kStageBytes = kQConsumers * JV * 16;
+    constexpr int kStageBytes = kQThreads * JV * 16;
     extern __shared__ __align__(128) unsigned char smem[];
     QShared &sh = *reinterpret_cast<QShared *>(smem + (size_t)kQStages * kStageBytes);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -488,26 +348,22 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
         for (int s = 0; s < kQStages; ++s) mbar_init(&sh.full[s], 1);
         sh.abort = 0;
         sh.nlist = 0;
-        sh.info.cmd = 0;
         mbar_init_fence();
     }
     __syncthreads();
-    if (warp == kQWarps) {
-        finalize_rows(a, sh, lane);
-        return;
-    }
 
     const int nvec = a.n / VEC;
     const uint32_t row_bytes = (uint32_t)nvec * 16u;
     int nj = JV;
     if (!FULL) {
-        nj = (nvec - tid + kQConsumers - 1) / kQConsumers;
+        nj = (nvec - tid + kQThreads - 1) / kQThreads;
         nj = nj < 0 ? 0 : (nj > JV ? JV : nj);
     }
     const T *base = reinterpret_cast<const T *>(a.logits) + a.vb;
     const ciar_quantify_out &o = a.out;
     const int64_t stride_rows = gridDim.x;
     const float inv_n = 1.0f / (float)a.n;
+    const bool per_row = a.radius_mode == CIAR_RADIUS_PER_ROW;
 
     // issues the copy of this CTA's k-th row into its stage (thread 0 only)
     auto issue = [&](int k) {
@@ -519,29 +375,57 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
             bulk_copy_g2s(smem + (size_t)s * kStageBytes, base + pr * a.row_stride, row_bytes, &sh.full[s]);
         }
     };
+    // the stored radius of this CTA's k-th row (every thread reads it, one row ahead of its use)
+    auto radius_of = [&](int k) -> float {
+        if (!per_row) return a.r_scalar;
+        const int64_t lr = blockIdx.x + (int64_t)k * stride_rows;
+        int64_t pr;
+        if (lr < a.rows && map_row(a.rm, lr, pr)) return reinterpret_cast<const float *>(a.radius)[pr];
+        return 0.f;
+    };
+    // a row whose list outgrew its slot: the slot's part joins the rest in the CTA's list (one warp)
+    auto finish_long = [&](Parked &p) {
+        for (int i = lane; i < kParkList; i += 32) sh.list[i] = p.list[i];
+        __syncwarp();
+        finish_row(a, p, sh.list, lane);
+        __syncwarp();
+        if (lane == 0) p.status = -1;  // done
+    };
+    // every warp finishes one parked row
+    auto finish_parked = [&](int count) {
+        __syncthreads();
+        if (warp < count) {
+            Parked &p = sh.park[warp];
+            if (p.status >= 0) {
+                if (p.nlist > kParkList) finish_long(p);
+                else finish_row(a, p, p.list, lane);
+            }
+        }
+        __syncthreads();
+    };
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < kQStages; ++s) issue(s);
     }
+    float rho_next = radius_of(0);
 
     uint32_t phases = 0;
-    int k = 0;
+    int k = 0, filled = 0;
     bool aborted = false;
     for (;; ++k) {
         const int64_t lr = blockIdx.x + (int64_t)k * stride_rows;
         if (lr >= a.rows) break;
         const int s = k % kQStages;
         int64_t pr;
-        if (!map_row(a.rm, lr, pr)) {  // a position past the end of the sequence: nothing to quantify
+        const bool active = map_row(a.rm, lr, pr);
+        const float rho = rho_next;
+        rho_next = radius_of(k + 1);
+        if (!active) {  // a position past the end of the sequence: nothing to quantify
             if (tid == 0) {
                 if (o.flag) o.flag[lr] = 0;
                 if (o.row_status) o.row_status[lr] = 0;
                 issue(k + kQStages);
             }
-            named_bar_sync(kBarFree, kQBlock);
-            if (tid == 0) sh.info.cmd = 2;
-            __syncwarp();
-            named_bar_arrive(kBarFull, kQBlock);
             continue;
         }
         const unsigned char *stage = smem + (size_t)s * kStageBytes;
@@ -552,28 +436,35 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
         typename V::Max mx = V::max_init();
 #pragma unroll
         for (int j = 0; j < JV; ++j)
-            if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * kQConsumers));
+            if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * kQThreads));
         const float tm = V::max_value(mx);
         const float wm = warp_redux_max(tm);
         if (lane == 0) sh.wmax[warp] = wm;
         if (tid == 0) {
             sh.argmin = INT_MAX;
             sh.nmax = 0;
+            sh.park[filled].nlist = 0;
         }
         __syncwarp();
-        named_bar_sync(kBarConsumers, kQConsumers);
+        named_bar_sync(kBarRow, kQThreads);
         if (sh.abort) {
             aborted = true;
             break;
+        }
+        if (filled > 0 && sh.park[filled - 1].nlist > kParkList && sh.park[filled - 1].status >= 0) {
+            // the row parked last listed more codes than its slot holds; the rest sits in the CTA's
+            // list, which this row is about to reuse: finish that row now
+            if (warp == 0) finish_long(sh.park[filled - 1]);
+            named_bar_sync(kBarRow, kQThreads);
         }
         const float m = warp_redux_max(sh.wmax[lane & (kQWarps - 1)]);
         if (tm == m) {  // this thread holds a maximum: its lowest index competes for the arg-max
             int best = INT_MAX;
             for (int j = nj - 1; j >= 0; --j) {
-                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQConsumers) * 16);
+                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
 #pragma unroll
                 for (int q = VEC - 1; q >= 0; --q)
-                    if (Elem<T>::widen(v[q]) == m) best = (tid + j * kQConsumers) * VEC + q;
+                    if (Elem<T>::widen(v[q]) == m) best = (tid + j * kQThreads) * VEC + q;
             }
             if (best != INT_MAX) atomicMin(&sh.argmin, best);
         }
@@ -588,13 +479,13 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
             for (int j = 0; j < JV; ++j) {
                 if (FULL || j < nj) {
                     float2 c[NPV];
-                    V::pairs(stage_vec(stage, tid + j * kQConsumers), c);
+                    V::pairs(stage_vec(stage, tid + j * kQThreads), c);
 #pragma unroll
                     for (int q = 0; q < NPV; ++q) {
                         const float2 d = __ffma2_rn(c[q], L2, nm2);
                         const float2 ev = make_float2(ex2_approx(d.x), ex2_approx(d.y));  // a NaN logit poisons the sums on purpose
                         z2 = __fadd2_rn(z2, ev);
-                        t2 = __ffma2_rn(ev, V::exponent_for_entropy(d), t2);
+                        t2 = __ffma2_rn(ev, d, t2);  // 0 * -inf = NaN for a -inf logit: redone below
                         e[j * NPV + q] = ev;
                     }
                 } else {
@@ -603,7 +494,20 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
                 }
             }
         }
-        float zs = z2.x + z2.y;
+        float zs = z2.x + z2.y, ts = t2.x + t2.y;
+        if (!(ts == ts)) {
+            // A -inf logit (exponential 0, exponent -inf) or a real NaN: form this thread's entropy sum
+            // again with the product of such a code taken as 0.  A real NaN still shows in the sum of exponentials.
+            ts = 0.f;
+            for (int j = 0; j < nj; ++j) {
+                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+#pragma unroll
+                for (int q = 0; q < VEC; ++q) {
+                    const float d = fmaf(Elem<T>::widen(v[q]), kLog2e, -m2);
+                    ts = fmaf(ex2_approx(d), fmaxf(d, kNegHuge), ts);
+                }
+            }
+        }
         const float e0 = ex2_approx(fmaf(m, kLog2e, -m2));  // the exponential every maximum got
         if (tm == m) {
             // This thread owns a maximum.  A term near 1 would cost the small terms their low bits, so its
@@ -620,10 +524,10 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
             zs = zz;
             atomicAdd(&sh.nmax, cnt);
         }
-        const float zt = warp_sum_pair(zs, t2.x + t2.y, lane);  // lanes 0..15: z, lanes 16..31: t
+        const float zt = warp_sum_pair(zs, ts, lane);  // lanes 0..15: z, lanes 16..31: t
         if (lane == 0) sh.wz[warp] = zt;
         __syncwarp();
-        named_bar_sync(kBarConsumers, kQConsumers);
+        named_bar_sync(kBarRow, kQThreads);
         float z = sh.wz[lane & (kQWarps - 1)];
 #pragma unroll
         for (int ofs = 8; ofs > 0; ofs >>= 1) z += __shfl_xor_sync(0xffffffffu, z, ofs);
@@ -631,14 +535,14 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
         z = fmaf((float)nmax, e0, z);
 
         int status = 0;
-        if (!(m > kLogitFloor) || !(z > 0.f) || !(z < INFINITY)) {
+        if (!(m > -INFINITY) || !(z > 0.f) || !(z < INFINITY)) {
             // an unusable row (NaN / +inf logit, no finite logit): classify it from the landed bytes
             // exactly as the row-status bits are defined
             if (tid == 0) sh.bad_nan = sh.bad_finite = 0;
-            named_bar_sync(kBarConsumers, kQConsumers);
+            named_bar_sync(kBarRow, kQThreads);
             int has_nan = 0, has_finite = 0;
             for (int j = 0; j < nj; ++j) {
-                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQConsumers) * 16);
+                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
 #pragma unroll
                 for (int q = 0; q < VEC; ++q) {
                     const float c = Elem<T>::widen(v[q]);
@@ -648,28 +552,30 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
             }
             if (has_nan) sh.bad_nan = 1;
             if (has_finite) sh.bad_finite = 1;
-            named_bar_sync(kBarConsumers, kQConsumers);
+            named_bar_sync(kBarRow, kQThreads);
             if (sh.bad_nan) status |= CIAR_ROW_NAN;
             if (!sh.bad_finite) status |= CIAR_ROW_NO_FINITE;
             if (!status) status = CIAR_ROW_NAN;  // sums overflowed without any single bad logit
         }
-        // the hand-off buffer (partial sums, list of large codes) and this row's constants are ours from here on
-        named_bar_sync(kBarFree, kQBlock);
-        const RowConst rc = sh.rc_tab[(k / kBatch) & 1][k % kBatch];
-        if (!(rc.rho == rc.rho)) status |= CIAR_ROW_NAN;
-        const bool direct = !status && !rc.series;
-        if (tid == 0 && !direct) {  // every consumer has read the stage: refill it
+        if (!(rho == rho)) status |= CIAR_ROW_NAN;
+        const float r = row_radius(rho, a.radius_is_raw, a.r_max);
+        const bool series = r <= 1.0f;
+        const bool direct = !status && !series;
+        if (tid == 0 && !direct) {  // every thread has read the stage: refill it
             fence_proxy_async_smem();
             issue(k + kQStages);
         }
+        Parked &pk = sh.park[filled];
 
         // ---- sweep 3: interval sums
-        const float c0 = z * inv_n, th = rc.theta_p * z;
-        if (!status && rc.series) {
-            // Codes above th are listed and clamped to th.  Most threads hold none, and a vector
-            // holding none is skipped on one comparison of its maximum.
-            const float e_tm = ex2_approx(fmaf(tm, kLog2e, -m2));  // this thread's largest exponential
-            if (__any_sync(0xffffffffu, e_tm > th)) {
+        const float c0 = z * inv_n, th = 0.00390625f * ex2_approx(-r * kLog2e) * z;  // clamp level: theta = 2^-8 e^-r
+        float r0 = 0.f, r1 = 0.f, r2 = 0.f;  // warp sums: r0, r1 hold two sums each (lanes 0..15 / 16..31)
+        if (!status && series) {
+            // Codes above th are listed and clamped to th.  Most threads hold none (seen from the thread's
+            // maximum logit), and a vector holding none is skipped on one comparison of its maximum.
+            // (th_log is a slightly low stand-in for log2(th), so the test on the thread's maximum errs on the safe side)
+            const float th_log = __log2f(th) - 1e-3f;
+            if (__builtin_expect(fmaf(tm, kLog2e, -m2) > th_log, 0)) {
 #pragma unroll
                 for (int j = 0; j < JV; ++j) {
                     float2 g = e[j * NPV];
@@ -677,19 +583,14 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
                     for (int q = 1; q < NPV; ++q) g = make_float2(fmaxf(g.x, e[j * NPV + q].x), fmaxf(g.y, e[j * NPV + q].y));
                     if (fmaxf(g.x, g.y) > th) {
 #pragma unroll
-                        for (int q = 0; q < NPV; ++q) {
-                            float2 ev = e[j * NPV + q];
-                            if (ev.x > th) {
-                                const int slot = atomicAdd(&sh.nlist, 1);
-                                if (slot < kListCap) sh.list[slot] = ev.x;
-                                ev.x = th;
+                        for (int q = 0; q < 2 * NPV; ++q) {
+                            float &ev = (q & 1) ? e[j * NPV + q / 2].y : e[j * NPV + q / 2].x;
+                            if (ev > th) {
+                                const int slot = atomicAdd(&pk.nlist, 1);
+                                if (slot < kParkList) pk.list[slot] = ev;
+                                else if (slot < kListCap) sh.list[slot] = ev;
+                                ev = th;
                             }
-                            if (ev.y > th) {
-                                const int slot = atomicAdd(&sh.nlist, 1);
-                                if (slot < kListCap) sh.list[slot] = ev.y;
-                                ev.y = th;
-                            }
-                            e[j * NPV + q] = ev;
                         }
                     }
                 }
@@ -707,26 +608,26 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
                     T4 = __ffma2_rn(y2, y2, T4);
                 }
             }
-            sh.part[0][tid] = T2.x + T2.y;
-            sh.part[1][tid] = T3.x + T3.y;
-            sh.part[2][tid] = T4.x + T4.y;
+            r0 = warp_sum_pair(T2.x + T2.y, T3.x + T3.y, lane);
+            r1 = warp_sum_f(T4.x + T4.y);
         } else if (direct) {
             // both bounds of every code, from the row still sitting in its stage
+            const DirectConst dc = make_direct_const(r, a.n);
             const float invz = 1.0f / z;
             float ps[5] = { 0.f, 0.f, 0.f, 0.f, 0.f };
 #pragma unroll 1
             for (int j = 0; j < nj; ++j) {
-                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQConsumers) * 16);
+                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
                 float c[VEC];
                 Elem<T>::load(v, c);
 #pragma unroll
                 for (int q = 0; q < VEC; ++q) {
                     const float ev = ex2_approx(fmaf(c[q], kLog2e, -m2));
                     const float x = ev * invz, sx = fmaf(-ev, invz, 1.0f);
-                    const float den_l = fmaf(rc.b1, sx, rc.a1), den_u = fmaf(rc.b1, x, rc.a1);
+                    const float den_l = fmaf(dc.b1, sx, dc.a1), den_u = fmaf(dc.b1, x, dc.a1);
                     const float xr = x * rcp_approx(den_l * den_u);
-                    const float pl = fmaf(xr * den_u, rc.a1, -rc.pl0);  // p^l term minus its centre
-                    const float dd = fmaf(xr, sx, -rc.dd0);             // width term minus its centre
+                    const float pl = fmaf(xr * den_u, dc.a1, -dc.pl0);  // p^l term minus its centre
+                    const float dd = fmaf(xr, sx, -dc.dd0);             // width term minus its centre
                     ps[0] += pl;
                     ps[1] += dd;
                     ps[2] = fmaf(pl, pl, ps[2]);
@@ -734,59 +635,65 @@ __global__ void __launch_bounds__(kQBlock, MINB) quantify_stream_kernel(const __
                     ps[4] = fmaf(dd, dd, ps[4]);
                 }
             }
-#pragma unroll
-            for (int q = 0; q < 5; ++q) {
-                const float w = warp_sum_f(ps[q]);
-                if (lane == 0) sh.dpart[q][warp] = w;
-            }
-            named_bar_sync(kBarConsumers, kQConsumers);
+            r0 = warp_sum_pair(ps[0], ps[1], lane);
+            r1 = warp_sum_pair(ps[2], ps[3], lane);
+            r2 = warp_sum_f(ps[4]);
+            named_bar_sync(kBarRow, kQThreads);
             if (tid == 0) {
                 fence_proxy_async_smem();
                 issue(k + kQStages);
             }
         }
 
-        // ---- hand the row to the finalizer warp
-        if (lane == 0) sh.info.zt[warp].x = zt;
-        if (lane == 16) sh.info.zt[warp].y = zt;
-        if (tid == 0) {
-            sh.info.lr = lr;
-            sh.info.pr = pr;
-            sh.info.m = m;
-            sh.info.e0 = e0;
-            sh.info.c0 = c0;
-            sh.info.th = th;
-            sh.info.argmin = sh.argmin;
-            sh.info.nmax = nmax;
-            sh.info.status = status;
-            sh.info.cmd = 0;
+        // ---- park the row's sums
+        if (lane == 0) {
+            pk.wsum[warp][0] = zt;
+            pk.wsum[warp][2] = r0;
+            pk.wsum[warp][4] = r1;
+            pk.wsum[warp][6] = r2;
         }
-        __syncwarp();
-        named_bar_arrive(kBarFull, kQBlock);
+        if (lane == 16) {
+            pk.wsum[warp][1] = zt;
+            pk.wsum[warp][3] = r0;
+            if (direct) pk.wsum[warp][5] = r1;
+        }
+        if (tid == 0) {
+            pk.lr = lr;
+            pk.pr = pr;
+            pk.m = m;
+            pk.e0 = e0;
+            pk.c0 = c0;
+            pk.th = th;
+            pk.rho = rho;
+            pk.r = r;
+            pk.argmin = sh.argmin;
+            pk.nmax = nmax;
+            pk.status = status;
+            pk.series = series;
+        }
+        if (++filled == kPark) {
+            finish_parked(filled);
+            filled = 0;
+        }
     }
+    if (filled > 0) finish_parked(filled);
 
-    if (aborted) {
+    if (aborted && tid == 0) {
         // A copy never arrived.  Mark this row and the rest of this CTA's rows, then give the
         // copies still in flight a last bounded chance to land before the CTA leaves.
-        if (tid == 0) {
-            for (int k2 = k;; ++k2) {
-                const int64_t lr = blockIdx.x + (int64_t)k2 * stride_rows;
-                if (lr >= a.rows) break;
-                write_unusable(o, lr, CIAR_ROW_TIMEOUT);
-            }
-            for (int s = 0; s < kQStages; ++s) mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kDrainCycles);
+        for (int k2 = k;; ++k2) {
+            const int64_t lr = blockIdx.x + (int64_t)k2 * stride_rows;
+            if (lr >= a.rows) break;
+            write_unusable(o, lr, CIAR_ROW_TIMEOUT);
         }
+        for (int s = 0; s < kQStages; ++s) mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kDrainCycles);
     }
-    named_bar_sync(kBarFree, kQBlock);
-    if (tid == 0) sh.info.cmd = 1;
-    __syncwarp();
-    named_bar_arrive(kBarFull, kQBlock);
 }
 
 template <typename T, int JV, int MINB, bool FULL>
 cudaError_t launch_one(const QuantifyArgs &a, cudaStream_t stream)
 {
-    constexpr size_t smem = (size_t)kQStages * kQConsumers * JV * 16 + sizeof(QShared);
+    constexpr size_t smem = (size_t)kQStages * kQThreads * JV * 16 + sizeof(QShared);
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
@@ -800,7 +707,7 @@ cudaError_t launch_one(const QuantifyArgs &a, cudaStream_t stream)
     }
     const int64_t cap = (int64_t)sm_count() * MINB;
     const unsigned grid = (unsigned)(a.rows < cap ? a.rows : cap);
-    quantify_stream_kernel<T, JV, MINB, FULL><<<grid, kQBlock, smem, stream>>>(a);
+    quantify_stream_kernel<T, JV, MINB, FULL><<<grid, kQThreads, smem, stream>>>(a);
     count_launch();
     return cudaGetLastError();
 }
@@ -809,7 +716,7 @@ template <typename T, int JV, int MINB>
 cudaError_t launch_jv(const QuantifyArgs &a, cudaStream_t stream)
 {
     const int nvec = a.n / Elem<T>::kVec;
-    if (nvec == kQConsumers * JV) return launch_one<T, JV, MINB, true>(a, stream);
+    if (nvec == kQThreads * JV) return launch_one<T, JV, MINB, true>(a, stream);
     return launch_one<T, JV, MINB, false>(a, stream);
 }
 
