@@ -179,6 +179,36 @@ ciar_status ciar_verify(const ciar_logits_desc *desc, const void *draft_logits, 
                         void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * ciar_verify without a workspace argument -- the paper has no counterpart; this entry point exists
+ * for integration reasons only.
+ *
+ * Some hosts of this library cannot give ciar_verify a workspace: a plug-in that runs inside another
+ * engine's pre-sized memory arena, a latency-critical serving loop, or code running between the
+ * begin and end of a stream capture must not call cudaMalloc (it may fail against the arena's
+ * budget, it synchronises the device, and it is illegal during capture), and some of them have no
+ * allocator of their own to carve a buffer from.  Here the scratch is a fixed array of
+ * CIAR_STATIC_SCRATCH_BYTES inside the library image: every GPU that loads the library holds that
+ * much memory until the process ends, whether or not this function is ever called.
+ *
+ * Same arguments, results and errors as ciar_verify, minus ws / ws_bytes, plus:
+ *   - WORKSPACE_TOO_SMALL when ciar_workspace_bytes(desc->rows, params->window) exceeds
+ *     CIAR_STATIC_SCRATCH_BYTES (2 MiB: enough for 120 000 rows at window 8); nothing is launched then.
+ *   - The first call on each device looks up the array's device address (once, with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - No cudaMalloc, cudaFree or other allocating call is made, on any call.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in
+ *     it; the part that must start at zero is cleared on the given stream at the start of every
+ *     call.  Two calls that may overlap on the GPU (different streams without an ordering between
+ *     them) race on it: order them, or use ciar_verify with separate workspaces.
+ */
+#define CIAR_STATIC_SCRATCH_BYTES (2 * 1024 * 1024)
+ciar_status ciar_verify_static(const ciar_logits_desc *desc, const void *draft_logits, const void *target_logits,
+                               const int32_t *draft_tokens, const uint8_t *flag,
+                               const float *draft_row_max, const float *draft_sum_exp,
+                               const float *u_accept, const float *u_resample,
+                               const ciar_verify_params *params, const ciar_verify_out *out, void *stream);
+
+/*
  * State of a batch of concurrent requests, all arrays device memory owned by the caller.
  *   pos int32[requests]: next position to generate; tokens_out int32[requests, seq_len];
  *   counters int64[8], accumulated over steps: 0 windows processed, 1 windows with a cloud call,

@@ -86,6 +86,9 @@ def load() -> ctypes.CDLL:
         lib.ciar_verify.argtypes = [ctypes.POINTER(LogitsDesc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                     ctypes.POINTER(VerifyParamsC), ctypes.POINTER(VerifyOutC), _vp,
                                     ctypes.c_size_t, _vp]
+        lib.ciar_verify_static.restype = ctypes.c_int
+        lib.ciar_verify_static.argtypes = [ctypes.POINTER(LogitsDesc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                           ctypes.POINTER(VerifyParamsC), ctypes.POINTER(VerifyOutC), _vp]
         lib.ciar_decode_init.restype = ctypes.c_int
         lib.ciar_decode_init.argtypes = [ctypes.POINTER(DecodeStateC), ctypes.c_int32, _vp]
         lib.ciar_decode_step.restype = ctypes.c_int
@@ -268,6 +271,30 @@ def verify(draft: torch.Tensor, target: torch.Tensor, draft_tokens: torch.Tensor
                             ctypes.byref(vp), ctypes.byref(oc), _ptr(workspace), workspace.numel(), _stream(stream))
     if st != 0:
         raise CiarError("ciar_verify", st)
+    return out
+
+
+STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
+
+
+def verify_static(draft: torch.Tensor, target: torch.Tensor, draft_tokens: torch.Tensor, flag: Optional[torch.Tensor],
+                  draft_row_max: Optional[torch.Tensor], draft_sum_exp: Optional[torch.Tensor],
+                  u_accept: torch.Tensor, u_resample: torch.Tensor, window: int, mode: int, out: VerifyOut,
+                  valid_begin: int = 0, valid_count: Optional[int] = None, stream=None) -> VerifyOut:
+    """ciar_verify_static: ciar_verify for callers that cannot provide a workspace (they may not
+    allocate device memory where they run).  The scratch is a fixed 2 MiB array inside the library,
+    shared by all calls on a device: calls that could overlap on the GPU must be ordered, and
+    batches whose workspace_bytes() exceeds STATIC_SCRATCH_BYTES are refused (status 4)."""
+    _require_cuda(draft, target, draft_tokens, flag, draft_row_max, draft_sum_exp, u_accept, u_resample)
+    if target.shape != draft.shape or target.dtype != draft.dtype or target.stride() != draft.stride():
+        raise ValueError("draft and target logits must share shape, dtype and strides")
+    desc = make_desc(draft, valid_begin, valid_count)
+    vp, oc = VerifyParamsC(window, mode), out.to_c()
+    st = load().ciar_verify_static(ctypes.byref(desc), _ptr(draft), _ptr(target), _ptr(draft_tokens), _ptr(flag),
+                                   _ptr(draft_row_max), _ptr(draft_sum_exp), _ptr(u_accept), _ptr(u_resample),
+                                   ctypes.byref(vp), ctypes.byref(oc), _stream(stream))
+    if st != 0:
+        raise CiarError("ciar_verify_static", st)
     return out
 
 
