@@ -124,4 +124,55 @@ __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b)
     return r;
 }
 
+// A 16-byte vector of a landed row.  fold_max() folds it into a running maximum (bf16: two packed
+// halves, NaN ignored), pairs() widens it to float2 pairs.
+template <typename T>
+struct Vec;
+
+template <>
+struct Vec<__nv_bfloat16> {
+    static constexpr int kPairs = 4;
+    typedef uint32_t Max;
+    static __device__ __forceinline__ Max max_init() { return 0xFF80FF80u; }  // (-inf, -inf)
+    static __device__ __forceinline__ Max fold_max(Max mx, const uint4 &v)
+    {
+        return bf16x2_max(mx, bf16x2_max(bf16x2_max(v.x, v.y), bf16x2_max(v.z, v.w)));
+    }
+    static __device__ __forceinline__ float max_value(Max mx)
+    {
+        const float2 p = unpack_bf16x2(mx);
+        return fmaxf(p.x, p.y);
+    }
+    static __device__ __forceinline__ void pairs(const uint4 &v, float2 (&c)[4])
+    {
+        c[0] = unpack_bf16x2(v.x);
+        c[1] = unpack_bf16x2(v.y);
+        c[2] = unpack_bf16x2(v.z);
+        c[3] = unpack_bf16x2(v.w);
+    }
+};
+
+template <>
+struct Vec<float> {
+    static constexpr int kPairs = 2;
+    typedef float Max;
+    static __device__ __forceinline__ Max max_init() { return -INFINITY; }
+    static __device__ __forceinline__ Max fold_max(Max mx, const uint4 &v)
+    {
+        return fmaxf(mx, fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)),
+                               fmaxf(__uint_as_float(v.z), __uint_as_float(v.w))));
+    }
+    static __device__ __forceinline__ float max_value(Max mx) { return mx; }
+    static __device__ __forceinline__ void pairs(const uint4 &v, float2 (&c)[2])
+    {
+        c[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+        c[1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
+    }
+};
+
+__device__ __forceinline__ const uint4 &stage_vec(const unsigned char *stage, int vi)
+{
+    return *reinterpret_cast<const uint4 *>(stage + (size_t)vi * 16);
+}
+
 }  // namespace ciar
