@@ -192,7 +192,7 @@ ciar_status ciar_verify(const ciar_logits_desc *desc, const void *draft_logits, 
  *
  * Same arguments, results and errors as ciar_verify, minus ws / ws_bytes, plus:
  *   - WORKSPACE_TOO_SMALL when ciar_workspace_bytes(desc->rows, params->window) exceeds
- *     CIAR_STATIC_SCRATCH_BYTES (2 MiB: enough for 120 000 rows at window 8); nothing is launched then.
+ *     CIAR_STATIC_SCRATCH_BYTES (2 MiB: enough for 72 000 rows at window 8); nothing is launched then.
  *   - The first call on each device looks up the array's device address (once, with that device
  *     current).  Make that first call outside any stream capture.
  *   - No cudaMalloc, cudaFree or other allocating call is made, on any call.

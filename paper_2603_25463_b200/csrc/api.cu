@@ -72,7 +72,7 @@ void fill_quantify_args(QuantifyArgs &a, const ciar_logits_desc *d, const void *
 
 // Layout of the workspace: verify scratch first, then the per-step arrays of the decode loop.
 struct WsLayout {
-    size_t window_done, candidate, accept;        // verify
+    size_t window_done, candidate, accept, tested, tq_max, tq_sum;  // verify
     size_t flag, row_max, sum_exp, first_flag, accepted_len, resampled;  // decode step
     size_t total;
 };
@@ -86,6 +86,9 @@ WsLayout ws_layout(int64_t rows, int32_t window)
     l.window_done = take(nw * 4);
     l.candidate = take(r * 4);
     l.accept = take(r);
+    l.tested = take((r + 1) * 4);
+    l.tq_max = take(r * 4);
+    l.tq_sum = take(r * 4);
     l.flag = take(r);
     l.row_max = take(r * 4);
     l.sum_exp = take(r * 4);
@@ -206,7 +209,12 @@ ciar_status ciar_verify(const ciar_logits_desc *desc, const void *draft_logits, 
     a.ws.window_done = reinterpret_cast<int32_t *>(w + l.window_done);
     a.ws.candidate = reinterpret_cast<int32_t *>(w + l.candidate);
     a.ws.accept = reinterpret_cast<uint8_t *>(w + l.accept);
+    a.ws.tested = reinterpret_cast<int32_t *>(w + l.tested);
+    a.ws.tq_max = reinterpret_cast<float *>(w + l.tq_max);
+    a.ws.tq_sum = reinterpret_cast<float *>(w + l.tq_sum);
     cudaStream_t st = (cudaStream_t)stream;
+    if (verify_stream_eligible(a, desc->dtype))
+        return launch_verify_stream(a, desc->dtype, st) == cudaSuccess ? CIAR_OK : CIAR_ERR_CUDA;
     if (cudaMemsetAsync(a.ws.window_done, 0, (size_t)(desc->rows / params->window) * 4, st) != cudaSuccess)
         return CIAR_ERR_CUDA;
     return launch_verify(a, desc->dtype, st) == cudaSuccess ? CIAR_OK : CIAR_ERR_CUDA;
@@ -293,6 +301,9 @@ ciar_status ciar_decode_step(const ciar_decode_state *state, const ciar_logits_d
     va.ws.window_done = reinterpret_cast<int32_t *>(w + l.window_done);
     va.ws.candidate = reinterpret_cast<int32_t *>(w + l.candidate);
     va.ws.accept = reinterpret_cast<uint8_t *>(w + l.accept);
+    va.ws.tested = reinterpret_cast<int32_t *>(w + l.tested);
+    va.ws.tq_max = reinterpret_cast<float *>(w + l.tq_max);
+    va.ws.tq_sum = reinterpret_cast<float *>(w + l.tq_sum);
     if (cudaMemsetAsync(va.ws.window_done, 0, (size_t)state->requests * 4, st) != cudaSuccess) return CIAR_ERR_CUDA;
     if (launch_verify(va, desc->dtype, st) != cudaSuccess) return CIAR_ERR_CUDA;
 

@@ -25,6 +25,9 @@ struct VerifyScratch {
     int32_t *window_done;  // [windows] arrival counters, zero before the launch
     int32_t *candidate;    // [rows] residual sample of each rejected row
     uint8_t *accept;       // [rows] accept bits when the caller did not ask for them
+    // streaming path only
+    int32_t *tested;       // [rows + 1] logical rows the cloud tests, in order; tested[rows] = how many
+    float *tq_max, *tq_sum;  // [rows] maximum and sum of exp(. - max) of the target rows that were tested
 };
 
 struct VerifyArgs {
@@ -56,6 +59,9 @@ cudaError_t launch_quantify(const QuantifyArgs &a, int dtype, cudaStream_t strea
 bool quantify_stream_eligible(const QuantifyArgs &a, int dtype);
 cudaError_t launch_quantify_stream(const QuantifyArgs &a, int dtype, cudaStream_t stream);
 cudaError_t launch_verify(const VerifyArgs &a, int dtype, cudaStream_t stream);
+// The streaming (plan, TMA-ring accept sweep, per-window finish) verifier and the test that says whether it covers a call.
+bool verify_stream_eligible(const VerifyArgs &a, int dtype);
+cudaError_t launch_verify_stream(const VerifyArgs &a, int dtype, cudaStream_t stream);
 cudaError_t launch_decode_init(const ciar_decode_state &st, int32_t pos0, cudaStream_t stream);
 cudaError_t launch_decode_update(const DecodeUpdateArgs &a, cudaStream_t stream);
 

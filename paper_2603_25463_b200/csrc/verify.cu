@@ -3,18 +3,11 @@
 // combine (first flag, accepted length, resampled token) done by whichever CTA of the window
 // finishes last -- no CTA ever waits for another.
 #include "ciar_internal.h"
+#include "verify_resample.cuh"
 
 namespace ciar {
 
 namespace {
-
-__device__ __forceinline__ float residual_term(float t, float c, float mq, float mp, float ratio)
-{
-    // exp(t - mq) - ratio * exp(c - mp) = zq * (q_i - p_i) with ratio = zq / zp
-    const float eq = ex2_approx((t - mq) * kLog2e);
-    const float ep = ex2_approx((c - mp) * kLog2e);
-    return fmaxf(fmaf(-ratio, ep, eq), 0.0f);
-}
 
 // First flagged row of a window (wlen if none).
 __device__ __forceinline__ int32_t first_flag_of(const uint8_t *flag, int64_t row0, int32_t wlen)
@@ -40,13 +33,11 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyArgs a)
     __shared__ double ds[2 * kWarps];
     __shared__ double scan_warp[kWarps];
     __shared__ double sh_d[4];
-    __shared__ int sh_i[4];
+    __shared__ int sh_i[4];  // 0: accept bit, 2..3: scratch of the resampler
     const T *dbase = reinterpret_cast<const T *>(a.draft);
     const T *tbase = reinterpret_cast<const T *>(a.target);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint8_t *accept_arr = a.out.accept ? a.out.accept : a.ws.accept;
-    if (threadIdx.x == 0) sh_i[2] = 0x7fffffff;
-    __syncthreads();
 
     for (int64_t lr = blockIdx.x; lr < a.rows; lr += gridDim.x) {
         const int64_t w = lr / a.window;
@@ -117,97 +108,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyArgs a)
                 }
 
                 if (!acc) {
-                    // residual sample: smallest k with cum_k > u * total, cum over max(0, q - p) in code order.
-                    // Thread t owns a contiguous run of vectors so that a block scan gives code-order prefixes.
-                    const float ratio = (float)(zq / zp);
-                    const int32_t nvec = rt.vec_end - rt.vec_begin;
-                    const int32_t vpt = (nvec + kThreads - 1) / kThreads;
-                    const int32_t v0 = rt.vec_begin + threadIdx.x * vpt;
-                    const int32_t v1 = min(v0 + vpt, rt.vec_end);
-                    double part = 0.0;
-                    for (int32_t vi = v0; vi < v1; ++vi) {
-                        float tv[V], cv[V];
-                        rt.load(vi, tv, -INFINITY);
-                        rd.load(vi, cv, -INFINITY);
-                        float s = 0.f;
-#pragma unroll
-                        for (int k = 0; k < V; ++k) s += residual_term(tv[k], cv[k], mq, mp, ratio);
-                        part += (double)s;
-                    }
-                    // inclusive block scan of the per-thread partials (double)
-                    double incl = part;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const double up = __shfl_up_sync(0xffffffffu, incl, o);
-                        if (lane >= o) incl += up;
-                    }
-                    if (lane == 31) scan_warp[warp] = incl;
-                    __syncthreads();
-                    double woff = 0.0, total = 0.0;
-#pragma unroll
-                    for (int ww = 0; ww < kWarps; ++ww) {
-                        if (ww < warp) woff += scan_warp[ww];
-                        total += scan_warp[ww];
-                    }
-                    incl += woff;
-                    // exclusive prefix = the previous thread's inclusive prefix, bit for bit, so that
-                    // the half-open intervals [excl, incl) tile [0, total) without gaps or overlaps
-                    double excl = __shfl_up_sync(0xffffffffu, incl, 1);
-                    if (lane == 0) excl = woff;
-                    if (threadIdx.x == 0) sh_i[1] = -1;
-                    __syncthreads();
-                    if (total > 0.0) {
-                        const double thr = (double)a.u_resample[pr] * total;
-                        // exactly one thread has excl <= thr < incl (threads with part == 0 never qualify)
-                        if (excl <= thr && thr < incl) {
-                            double cum = excl;
-                            int32_t pick = -1, last_pos = -1;
-                            for (int32_t vi = v0; vi < v1 && pick < 0; ++vi) {
-                                float tv[V], cv[V], rs[V];
-                                const int32_t i0 = rt.load(vi, tv, -INFINITY);
-                                rd.load(vi, cv, -INFINITY);
-                                float s = 0.f;
-#pragma unroll
-                                for (int k = 0; k < V; ++k) {
-                                    rs[k] = residual_term(tv[k], cv[k], mq, mp, ratio);
-                                    s += rs[k];
-                                }
-                                if (cum + (double)s > thr) {
-                                    double c2 = cum;
-#pragma unroll
-                                    for (int k = 0; k < V; ++k) {
-                                        if (rs[k] > 0.f) last_pos = i0 + k;
-                                        c2 += (double)rs[k];
-                                        if (pick < 0 && rs[k] > 0.f && c2 > thr) pick = i0 + k;
-                                    }
-                                    if (pick < 0) pick = last_pos;  // rounding: the crossing is at the vector's end
-                                } else {
-                                    cum += (double)s;
-#pragma unroll
-                                    for (int k = 0; k < V; ++k)
-                                        if (rs[k] > 0.f) last_pos = i0 + k;
-                                }
-                            }
-                            if (pick < 0) pick = last_pos;
-                            sh_i[1] = pick;
-                        }
-                        __syncthreads();
-                        cand = sh_i[1] >= 0 ? sh_i[1] + a.vb : -1;
-                    } else {
-                        // p == q wherever q > 0: fall back to the mode of q (lowest index at the maximum)
-                        int32_t amin = 0x7fffffff;
-                        for (int32_t vi = rt.vec_begin + threadIdx.x; vi < rt.vec_end; vi += kThreads) {
-                            float tv[V];
-                            const int32_t i0 = rt.load(vi, tv, -INFINITY);
-#pragma unroll
-                            for (int k = 0; k < V; ++k)
-                                if (tv[k] == mq) amin = min(amin, i0 + k);
-                        }
-                        atomicMin(&sh_i[2], amin);  // sh_i[2] is reset below before use
-                        __syncthreads();
-                        cand = sh_i[2] + a.vb;
-                    }
-                    __syncthreads();
+                    cand = resample_row(rd, rt, mp, zp, mq, zq, a.u_resample[pr], a.vb, scan_warp, sh_i + 2);
                 }
             }
         }
@@ -248,7 +149,6 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyArgs a)
                 if (a.out.cloud_call) a.out.cloud_call[w] = (uint8_t)(f < wlen);
                 a.ws.window_done[w] = 0;  // ready for the next launch
             }
-            sh_i[2] = 0x7fffffff;
         }
         __syncthreads();
     }

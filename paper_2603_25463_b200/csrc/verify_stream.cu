@@ -1,0 +1,462 @@
+// Streaming verifier for rows that fit on chip (2048 .. 16384 codes) when the draft rows' softmax
+// statistics come with the call.  Three launches, none of which waits for another CTA:
+//   plan    one CTA: per window the first flagged row and which rows the cloud tests; the tested
+//           rows are written out as one compact list, so that the next kernel's CTAs get equal shares.
+//   accept  persistent CTAs walk the list; target rows arrive through a ring of shared-memory
+//           stages filled by bulk (TMA) copies; two sweeps (maximum, sum of exponentials); every 16
+//           rows each warp finishes one row: the accept test on the drafted token, in double.
+//   window  one CTA per window: accepted length, and for a rejected window the residual sample.
+#include <climits>
+
+#include "ciar_internal.h"
+#include "stream_common.cuh"
+#include "verify_resample.cuh"
+
+namespace ciar {
+
+namespace {
+
+constexpr int kVThreads = 512;
+constexpr int kVWarps = kVThreads / 32;
+constexpr int kVStages = 3;
+constexpr int kVPark = 16;
+constexpr int kPlanThreads = 1024;
+constexpr long long kWaitCycles = 2000000000ll;
+constexpr long long kDrainCycles = 20000000ll;
+
+__device__ __forceinline__ bool tested_row(int mode, int32_t j, int32_t f, int32_t wlen, const uint8_t *flag, int64_t lr)
+{
+    if (j >= wlen) return false;
+    if (mode == CIAR_VERIFY_ALL) return true;
+    if (mode == CIAR_VERIFY_ANCHORED) return j >= f;
+    return flag[lr] != 0;
+}
+
+// ---- plan
+__global__ void __launch_bounds__(kPlanThreads) verify_plan_kernel(VerifyArgs a)
+{
+    __shared__ int warp_tot[kPlanThreads / 32];
+    __shared__ int base_sh;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t nw = a.rows / a.window;
+    uint8_t *accept_arr = a.out.accept ? a.out.accept : a.ws.accept;
+    if (tid == 0) base_sh = 0;
+    __syncthreads();
+    for (int64_t w0 = 0; w0 < nw; w0 += kPlanThreads) {
+        const int64_t w = w0 + tid;
+        int cnt = 0;
+        int32_t f = 0, wlen = 0;
+        if (w < nw) {
+            wlen = window_len(a.rm, w);
+            const int64_t row0 = w * a.window;
+            f = wlen;
+            if (a.mode == CIAR_VERIFY_ALL) {
+                f = 0;
+            } else {
+                for (int32_t j = 0; j < wlen; ++j)
+                    if (a.flag[row0 + j]) { f = j; break; }
+            }
+            if (a.out.first_flag) a.out.first_flag[w] = f;
+            if (a.out.cloud_call) a.out.cloud_call[w] = (uint8_t)(f < wlen);
+            for (int32_t j = 0; j < a.window; ++j) {
+                const int64_t lr = row0 + j;
+                if (tested_row(a.mode, j, f, wlen, a.flag, lr)) {
+                    ++cnt;
+                } else {  // rows the cloud does not test count as kept
+                    accept_arr[lr] = 1;
+                    if (a.out.p_draft_tok) a.out.p_draft_tok[lr] = 0.f;
+                    if (a.out.p_target_tok) a.out.p_target_tok[lr] = 0.f;
+                    if (a.out.row_status) a.out.row_status[lr] = 0;
+                }
+            }
+        }
+        // exclusive scan of cnt over the CTA
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        int woff = 0, total = 0;
+        for (int ww = 0; ww < kPlanThreads / 32; ++ww) {
+            if (ww < warp) woff += warp_tot[ww];
+            total += warp_tot[ww];
+        }
+        int pos = base_sh + woff + incl - cnt;
+        if (w < nw) {
+            const int64_t row0 = w * a.window;
+            for (int32_t j = 0; j < a.window; ++j)
+                if (tested_row(a.mode, j, f, wlen, a.flag, row0 + j)) a.ws.tested[pos++] = (int32_t)(row0 + j);
+        }
+        __syncthreads();
+        if (tid == 0) base_sh += total;
+        __syncthreads();
+    }
+    if (tid == 0) a.ws.tested[a.rows] = base_sh;
+}
+
+// ---- accept
+
+// Softmax statistics and status bits of one row straight from global memory, by one warp (the
+// slow way: only rows whose streamed statistics came out unusable take it).
+template <typename T>
+__device__ __noinline__ int warp_row_stats(const T *row, int32_t n, int lane, float &m_out, double &z_out)
+{
+    float m = -INFINITY;
+    int has_nan = 0, has_finite = 0;
+    for (int32_t i = lane; i < n; i += 32) {
+        const float c = Elem<T>::widen(row[i]);
+        if (!(c == c) || c == INFINITY) has_nan = 1;
+        if (c == c && fabsf(c) != INFINITY) has_finite = 1;
+        m = fmaxf(m, c);
+    }
+    m = warp_redux_max(m);
+    has_nan = __any_sync(0xffffffffu, has_nan);
+    has_finite = __any_sync(0xffffffffu, has_finite);
+    int status = 0;
+    if (has_nan) status |= CIAR_ROW_NAN;
+    if (!has_finite) status |= CIAR_ROW_NO_FINITE;
+    double z = 0.0;
+    if (!status) {
+        for (int32_t i = lane; i < n; i += 32) z += (double)ex2_approx((Elem<T>::widen(row[i]) - m) * kLog2e);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    }
+    m_out = m;
+    z_out = z;
+    return status;
+}
+
+struct VParked {
+    float wz[kVWarps];  // per-warp sums of exp(t - m) (terms equal to e0 left out)
+    int64_t lr;
+    float m, e0;
+    int nmax;
+};
+
+struct VShared {
+    unsigned long long full[kVStages];
+    float wmax[kVWarps];
+    int nmax, abort;
+    VParked park[kVPark];
+};
+
+// The accept test of one tested row, by one warp: u * p_x < q_x in double, p and q the draft's
+// and the target's probability of the drafted token.
+template <typename T>
+__device__ __noinline__ void accept_row(const VerifyArgs &a, const VParked &pk, int lane)
+{
+    const int64_t lr = pk.lr;
+    int64_t pr;
+    map_row(a.rm, lr, pr);
+    const T *drow = reinterpret_cast<const T *>(a.draft) + pr * a.row_stride + a.vb;
+    const T *trow = reinterpret_cast<const T *>(a.target) + pr * a.row_stride + a.vb;
+    // target statistics from the sweeps
+    double zq = lane < kVWarps ? (double)pk.wz[lane] : 0.0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) zq += __shfl_xor_sync(0xffffffffu, zq, o);
+    zq += (double)pk.nmax * (double)pk.e0;
+    float mq = pk.m;
+    // the exponent used was c * log2e_f - fl(m * log2e_f): take the common offset out again
+    const double off = (double)mq * (double)kLog2e - (double)(mq * kLog2e);
+    zq *= exp2(-off);
+    int status = 0;
+    if (!(mq > -INFINITY) || !(zq > 0.0) || !(zq < INFINITY)) status |= warp_row_stats(trow, a.n, lane, mq, zq);
+    // draft statistics from the quantifier; unusable ones are recomputed to learn what is wrong with the row
+    float mp = a.draft_row_max[lr];
+    double zp = (double)a.draft_sum_exp[lr];
+    if (!(zp > 0.0) || !(zp < INFINITY) || !(mp == mp)) status |= warp_row_stats(drow, a.n, lane, mp, zp);
+    if (lane != 0) return;
+    const int32_t x = a.tokens[pr];
+    const bool bad_token = (x < 0 || x >= a.vocab);
+    if (bad_token) status |= CIAR_ROW_BAD_TOKEN;
+    int acc = 0;
+    float px_out = __int_as_float(0x7fc00000), qx_out = px_out;
+    if (!(status & (CIAR_ROW_NAN | CIAR_ROW_NO_FINITE))) {
+        double px = 0.0, qx = 0.0;
+        if (x >= a.vb && x < a.vb + a.n) {  // a code outside the valid slice has probability 0
+            const double cx = (double)Elem<T>::widen(drow[x - a.vb]);
+            const double tx = (double)Elem<T>::widen(trow[x - a.vb]);
+            px = exp(cx - (double)mp) / zp;
+            qx = exp(tx - (double)mq) / zq;
+        }
+        acc = (!bad_token && (double)a.u_accept[pr] * px < qx) ? 1 : 0;
+        if (!bad_token) {
+            px_out = (float)px;
+            qx_out = (float)qx;
+        }
+        a.ws.tq_max[lr] = mq;
+        a.ws.tq_sum[lr] = (float)zq;
+    } else {
+        a.ws.tq_max[lr] = mq;
+        a.ws.tq_sum[lr] = __int_as_float(0x7fc00000);  // tells the window kernel that there is nothing to resample from
+    }
+    uint8_t *accept_arr = a.out.accept ? a.out.accept : a.ws.accept;
+    accept_arr[lr] = (uint8_t)acc;
+    if (a.out.p_draft_tok) a.out.p_draft_tok[lr] = px_out;
+    if (a.out.p_target_tok) a.out.p_target_tok[lr] = qx_out;
+    if (a.out.row_status) a.out.row_status[lr] = (uint8_t)status;
+}
+
+template <typename T, int JV, bool FULL>
+__global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __grid_constant__ VerifyArgs a)
+{
+    typedef Vec<T> V;
+    constexpr int VEC = Elem<T>::kVec;
+    constexpr int NPV = V::kPairs;
+    constexpr int kStageBytes = kVThreads * JV * 16;
+    extern __shared__ __align__(128) unsigned char smem[];
+    VShared &sh = *reinterpret_cast<VShared *>(smem + (size_t)kVStages * kStageBytes);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+#pragma unroll
+        for (int s = 0; s < kVStages; ++s) mbar_init(&sh.full[s], 1);
+        sh.abort = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+    const int nvec = a.n / VEC;
+    const uint32_t row_bytes = (uint32_t)nvec * 16u;
+    int nj = JV;
+    if (!FULL) {
+        nj = (nvec - tid + kVThreads - 1) / kVThreads;
+        nj = nj < 0 ? 0 : (nj > JV ? JV : nj);
+    }
+    const T *tbase = reinterpret_cast<const T *>(a.target) + a.vb;
+    const int total = a.ws.tested[a.rows];  // written by the plan kernel
+    const int stride = gridDim.x;
+
+    auto issue = [&](int k) {  // thread 0: copy this CTA's k-th tested row into its stage
+        const int idx = blockIdx.x + k * stride;
+        if (idx < total) {
+            int64_t pr;
+            map_row(a.rm, a.ws.tested[idx], pr);
+            const int s = k % kVStages;
+            mbar_arrive_expect_tx(&sh.full[s], row_bytes);
+            bulk_copy_g2s(smem + (size_t)s * kStageBytes, tbase + pr * a.row_stride, row_bytes, &sh.full[s]);
+        }
+    };
+    auto finish_parked = [&](int count) {
+        __syncthreads();
+        if (warp < count) accept_row<T>(a, sh.park[warp], lane);
+        __syncthreads();
+    };
+    if (tid == 0) {
+#pragma unroll
+        for (int s = 0; s < kVStages; ++s) issue(s);
+    }
+    uint32_t phases = 0;
+    int k = 0, filled = 0;
+    bool aborted = false;
+    for (;; ++k) {
+        const int idx = blockIdx.x + k * stride;
+        if (idx >= total) break;
+        const int s = k % kVStages;
+        const unsigned char *stage = smem + (size_t)s * kStageBytes;
+        if (mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kWaitCycles)) phases ^= 1u << s;
+        else sh.abort = 1;
+        // sweep 1: maximum
+        typename V::Max mx = V::max_init();
+#pragma unroll
+        for (int j = 0; j < JV; ++j)
+            if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * kVThreads));
+        const float tm = V::max_value(mx);
+        const float wm = warp_redux_max(tm);
+        if (lane == 0) sh.wmax[warp] = wm;
+        if (tid == 0) sh.nmax = 0;
+        __syncwarp();
+        __syncthreads();
+        if (sh.abort) {
+            aborted = true;
+            break;
+        }
+        const float m = warp_redux_max(sh.wmax[lane & (kVWarps - 1)]);
+        // sweep 2: sum of exponentials; terms equal to the maximum's are counted, not summed
+        const float m2 = m * kLog2e;
+        const float e0 = ex2_approx(fmaf(m, kLog2e, -m2));
+        float2 z2 = f2(0.f);
+        {
+            const float2 L2 = f2(kLog2e), nm2 = f2(-m2);
+#pragma unroll
+            for (int j = 0; j < JV; ++j) {
+                if (FULL || j < nj) {
+                    float2 c[NPV];
+                    V::pairs(stage_vec(stage, tid + j * kVThreads), c);
+#pragma unroll
+                    for (int q = 0; q < NPV; ++q) {
+                        const float2 d = __ffma2_rn(c[q], L2, nm2);
+                        z2 = __fadd2_rn(z2, make_float2(ex2_approx(d.x), ex2_approx(d.y)));
+                    }
+                }
+            }
+        }
+        float zs = z2.x + z2.y;
+        if (tm == m) {  // redo this thread's sum without the maxima (kept exactly, as a count)
+            float zz = 0.f;
+            int cnt = 0;
+            for (int j = 0; j < nj; ++j) {
+                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kVThreads) * 16);
+#pragma unroll
+                for (int q = 0; q < VEC; ++q) {
+                    const float ev = ex2_approx(fmaf(Elem<T>::widen(v[q]), kLog2e, -m2));
+                    if (ev == e0) ++cnt; else zz += ev;
+                }
+            }
+            zs = zz;
+            atomicAdd(&sh.nmax, cnt);
+        }
+        const float wz = warp_sum_f(zs);
+        VParked &pk = sh.park[filled];
+        if (lane == 0) pk.wz[warp] = wz;
+        __syncthreads();  // every thread has read the stage, the count of maxima is complete
+        if (tid == 0) {
+            fence_proxy_async_smem();
+            issue(k + kVStages);
+            pk.lr = a.ws.tested[idx];
+            pk.m = m;
+            pk.e0 = e0;
+            pk.nmax = sh.nmax;
+        }
+        if (++filled == kVPark) {
+            finish_parked(filled);
+            filled = 0;
+        }
+    }
+    if (filled > 0) finish_parked(filled);
+    if (aborted && tid == 0) {
+        // A copy never arrived: the rows this CTA still owed are marked, and the copies in flight
+        // get a last bounded chance to land before the CTA leaves.
+        uint8_t *accept_arr = a.out.accept ? a.out.accept : a.ws.accept;
+        for (int k2 = k;; ++k2) {
+            const int idx = blockIdx.x + k2 * stride;
+            if (idx >= total) break;
+            const int64_t lr = a.ws.tested[idx];
+            accept_arr[lr] = 0;
+            a.ws.tq_sum[lr] = __int_as_float(0x7fc00000);
+            if (a.out.row_status) a.out.row_status[lr] = CIAR_ROW_TIMEOUT;
+        }
+        for (int s = 0; s < kVStages; ++s) mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kDrainCycles);
+    }
+}
+
+// ---- window: accepted length and, for a rejected window, the residual sample of its first rejected row
+template <typename T>
+__global__ void __launch_bounds__(kThreads) verify_window_kernel(VerifyArgs a)
+{
+    __shared__ double scan_warp[kWarps];
+    __shared__ int sh_i[2];
+    __shared__ int sh_a;
+    const T *dbase = reinterpret_cast<const T *>(a.draft);
+    const T *tbase = reinterpret_cast<const T *>(a.target);
+    const uint8_t *accept_arr = a.out.accept ? a.out.accept : a.ws.accept;
+    const int64_t nw = a.rows / a.window;
+    for (int64_t w = blockIdx.x; w < nw; w += gridDim.x) {
+        const int32_t wlen = window_len(a.rm, w);
+        const int64_t row0 = w * a.window;
+        if (threadIdx.x == 0) {
+            int32_t f = 0;
+            if (a.mode != CIAR_VERIFY_ALL) {
+                f = wlen;
+                for (int32_t j = 0; j < wlen; ++j)
+                    if (a.flag[row0 + j]) { f = j; break; }
+            }
+            int32_t acc_len = wlen;
+            for (int32_t j = 0; j < wlen; ++j)
+                if (tested_row(a.mode, j, f, wlen, a.flag, row0 + j) && accept_arr[row0 + j] == 0) { acc_len = j; break; }
+            sh_a = acc_len;
+            if (a.out.accepted_len) a.out.accepted_len[w] = acc_len;
+        }
+        __syncthreads();
+        const int32_t acc_len = sh_a;
+        int32_t tok = -1;
+        if (acc_len < wlen) {
+            const int64_t lr = row0 + acc_len;
+            int64_t pr;
+            map_row(a.rm, lr, pr);
+            const float mq = a.ws.tq_max[lr];
+            const double zq = (double)a.ws.tq_sum[lr];
+            const float mp = a.draft_row_max[lr];
+            const double zp = (double)a.draft_sum_exp[lr];
+            // unusable logits on either side (their statistics are NaN): nothing to resample from
+            if (zq > 0.0 && zq < INFINITY && zp > 0.0 && zp < INFINITY && mp == mp) {
+                const RowView<T> rd(dbase + pr * a.row_stride, a.vb, a.n);
+                const RowView<T> rt(tbase + pr * a.row_stride, a.vb, a.n);
+                tok = resample_row(rd, rt, mp, zp, mq, zq, a.u_resample[pr], a.vb, scan_warp, sh_i);
+            }
+        }
+        if (threadIdx.x == 0) {
+            if (a.out.resampled_token) a.out.resampled_token[w] = tok;
+            a.ws.candidate[row0] = tok;  // kept for the decode step, which reads its result here
+        }
+        __syncthreads();
+    }
+}
+
+template <typename T, int JV>
+cudaError_t launch_accept(const VerifyArgs &a, cudaStream_t stream, bool full)
+{
+    constexpr size_t smem = (size_t)kVStages * kVThreads * JV * 16 + sizeof(VShared);
+    static bool configured[64][2] = {};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev][full]) {
+        err = full ? cudaFuncSetAttribute(verify_accept_kernel<T, JV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                   : cudaFuncSetAttribute(verify_accept_kernel<T, JV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        configured[dev][full] = true;
+    }
+    const int64_t cap = (int64_t)sm_count() * 2;
+    const unsigned grid = (unsigned)(a.rows < cap ? a.rows : cap);
+    if (full) verify_accept_kernel<T, JV, true><<<grid, kVThreads, smem, stream>>>(a);
+    else verify_accept_kernel<T, JV, false><<<grid, kVThreads, smem, stream>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_all(const VerifyArgs &a, cudaStream_t stream)
+{
+    verify_plan_kernel<<<1, kPlanThreads, 0, stream>>>(a);
+    count_launch();
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    const int nvec = a.n / Elem<T>::kVec;
+    const int jv = nvec <= kVThreads ? 1 : (nvec <= 2 * kVThreads ? 2 : (nvec <= 4 * kVThreads ? 4 : 8));
+    const bool full = nvec == kVThreads * jv;
+    switch (jv) {
+    case 1: err = launch_accept<T, 1>(a, stream, full); break;
+    case 2: err = launch_accept<T, 2>(a, stream, full); break;
+    case 4: err = launch_accept<T, 4>(a, stream, full); break;
+    default: err = launch_accept<T, 8>(a, stream, full); break;
+    }
+    if (err != cudaSuccess) return err;
+    const int64_t nw = a.rows / a.window;
+    const int64_t cap = (int64_t)sm_count() * 8;
+    const unsigned grid = (unsigned)(nw < cap ? nw : cap);
+    verify_window_kernel<T><<<grid, kThreads, 0, stream>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool verify_stream_eligible(const VerifyArgs &a, int dtype)
+{
+    const int vec = dtype == CIAR_F32 ? 4 : 8;
+    if (!a.draft_row_max || !a.draft_sum_exp) return false;
+    if (a.vb % vec != 0 || a.n % vec != 0) return false;
+    if (a.rows >= INT_MAX) return false;
+    return a.n >= 2048 && a.n <= 16384;
+}
+
+cudaError_t launch_verify_stream(const VerifyArgs &a, int dtype, cudaStream_t stream)
+{
+    if (a.rows == 0) return cudaSuccess;
+    return dtype == CIAR_F32 ? launch_all<float>(a, stream) : launch_all<__nv_bfloat16>(a, stream);
+}
+
+}  // namespace ciar
