@@ -304,8 +304,12 @@ ciar_status ciar_decode_step(const ciar_decode_state *state, const ciar_logits_d
     va.ws.tested = reinterpret_cast<int32_t *>(w + l.tested);
     va.ws.tq_max = reinterpret_cast<float *>(w + l.tq_max);
     va.ws.tq_sum = reinterpret_cast<float *>(w + l.tq_sum);
-    if (cudaMemsetAsync(va.ws.window_done, 0, (size_t)state->requests * 4, st) != cudaSuccess) return CIAR_ERR_CUDA;
-    if (launch_verify(va, desc->dtype, st) != cudaSuccess) return CIAR_ERR_CUDA;
+    if (verify_stream_eligible(va, desc->dtype)) {
+        if (launch_verify_stream(va, desc->dtype, st) != cudaSuccess) return CIAR_ERR_CUDA;
+    } else {
+        if (cudaMemsetAsync(va.ws.window_done, 0, (size_t)state->requests * 4, st) != cudaSuccess) return CIAR_ERR_CUDA;
+        if (launch_verify(va, desc->dtype, st) != cudaSuccess) return CIAR_ERR_CUDA;
+    }
 
     DecodeUpdateArgs ua;
     ua.st = *state;
