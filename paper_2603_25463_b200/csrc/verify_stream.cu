@@ -1,6 +1,6 @@
 // Streaming verifier for rows that fit on chip (2048 .. 16384 codes) when the draft rows' softmax
 // statistics come with the call.  Three launches, none of which waits for another CTA:
-//   plan    one CTA: per window the first flagged row and which rows the cloud tests; the tested
+//   plan    one thread per window: the first flagged row and which rows the cloud tests; the tested
 //           rows are written out as one compact list, so that the next kernel's CTAs get equal shares.
 //   accept  persistent CTAs walk the list; target rows arrive through a ring of shared-memory
 //           stages filled by bulk (TMA) copies; two sweeps (maximum, sum of exponentials); every 16
@@ -20,7 +20,7 @@ constexpr int kVThreads = 512;
 constexpr int kVWarps = kVThreads / 32;
 constexpr int kVStages = 3;
 constexpr int kVPark = 16;
-constexpr int kPlanThreads = 1024;
+constexpr int kPlanThreads = 128;
 constexpr long long kWaitCycles = 2000000000ll;
 constexpr long long kDrainCycles = 20000000ll;
 
@@ -33,68 +33,52 @@ __device__ __forceinline__ bool tested_row(int mode, int32_t j, int32_t f, int32
 }
 
 // ---- plan
+// One thread per window.  A warp reserves room for its windows' tested rows with one atomic add on
+// the list's counter (tested[rows], zeroed before the launch); the order of the list is not fixed
+// from run to run, and nothing depends on it.
 __global__ void __launch_bounds__(kPlanThreads) verify_plan_kernel(VerifyArgs a)
 {
-    __shared__ int warp_tot[kPlanThreads / 32];
-    __shared__ int base_sh;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int lane = threadIdx.x & 31;
     const int64_t nw = a.rows / a.window;
+    const int64_t w = (int64_t)blockIdx.x * kPlanThreads + threadIdx.x;
     uint8_t *accept_arr = a.out.accept ? a.out.accept : a.ws.accept;
-    if (tid == 0) base_sh = 0;
-    __syncthreads();
-    for (int64_t w0 = 0; w0 < nw; w0 += kPlanThreads) {
-        const int64_t w = w0 + tid;
-        int cnt = 0;
-        int32_t f = 0, wlen = 0;
-        if (w < nw) {
-            wlen = window_len(a.rm, w);
-            const int64_t row0 = w * a.window;
+    int cnt = 0;
+    int32_t f = 0, wlen = 0;
+    const int64_t row0 = w * a.window;
+    if (w < nw) {
+        wlen = window_len(a.rm, w);
+        if (a.mode != CIAR_VERIFY_ALL) {
             f = wlen;
-            if (a.mode == CIAR_VERIFY_ALL) {
-                f = 0;
-            } else {
-                for (int32_t j = 0; j < wlen; ++j)
-                    if (a.flag[row0 + j]) { f = j; break; }
-            }
-            if (a.out.first_flag) a.out.first_flag[w] = f;
-            if (a.out.cloud_call) a.out.cloud_call[w] = (uint8_t)(f < wlen);
-            for (int32_t j = 0; j < a.window; ++j) {
-                const int64_t lr = row0 + j;
-                if (tested_row(a.mode, j, f, wlen, a.flag, lr)) {
-                    ++cnt;
-                } else {  // rows the cloud does not test count as kept
-                    accept_arr[lr] = 1;
-                    if (a.out.p_draft_tok) a.out.p_draft_tok[lr] = 0.f;
-                    if (a.out.p_target_tok) a.out.p_target_tok[lr] = 0.f;
-                    if (a.out.row_status) a.out.row_status[lr] = 0;
-                }
+            for (int32_t j = wlen - 1; j >= 0; --j)  // independent loads, lowest flagged row wins
+                if (a.flag[row0 + j]) f = j;
+        }
+        if (a.out.first_flag) a.out.first_flag[w] = f;
+        if (a.out.cloud_call) a.out.cloud_call[w] = (uint8_t)(f < wlen);
+        for (int32_t j = 0; j < a.window; ++j) {
+            const int64_t lr = row0 + j;
+            if (tested_row(a.mode, j, f, wlen, a.flag, lr)) {
+                ++cnt;
+            } else {  // rows the cloud does not test count as kept
+                accept_arr[lr] = 1;
+                if (a.out.p_draft_tok) a.out.p_draft_tok[lr] = 0.f;
+                if (a.out.p_target_tok) a.out.p_target_tok[lr] = 0.f;
+                if (a.out.row_status) a.out.row_status[lr] = 0;
             }
         }
-        // exclusive scan of cnt over the CTA
-        int incl = cnt;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
-        }
-        if (lane == 31) warp_tot[warp] = incl;
-        __syncthreads();
-        int woff = 0, total = 0;
-        for (int ww = 0; ww < kPlanThreads / 32; ++ww) {
-            if (ww < warp) woff += warp_tot[ww];
-            total += warp_tot[ww];
-        }
-        int pos = base_sh + woff + incl - cnt;
-        if (w < nw) {
-            const int64_t row0 = w * a.window;
-            for (int32_t j = 0; j < a.window; ++j)
-                if (tested_row(a.mode, j, f, wlen, a.flag, row0 + j)) a.ws.tested[pos++] = (int32_t)(row0 + j);
-        }
-        __syncthreads();
-        if (tid == 0) base_sh += total;
-        __syncthreads();
     }
-    if (tid == 0) a.ws.tested[a.rows] = base_sh;
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    int base = 0;
+    if (lane == 31 && incl > 0) base = atomicAdd(&a.ws.tested[a.rows], incl);
+    base = __shfl_sync(0xffffffffu, base, 31);
+    int pos = base + incl - cnt;
+    if (w < nw)
+        for (int32_t j = 0; j < a.window; ++j)
+            if (tested_row(a.mode, j, f, wlen, a.flag, row0 + j)) a.ws.tested[pos++] = (int32_t)(row0 + j);
 }
 
 // ---- accept
@@ -420,9 +404,12 @@ cudaError_t launch_accept(const VerifyArgs &a, cudaStream_t stream, bool full)
 template <typename T>
 cudaError_t launch_all(const VerifyArgs &a, cudaStream_t stream)
 {
-    verify_plan_kernel<<<1, kPlanThreads, 0, stream>>>(a);
+    cudaError_t err = cudaMemsetAsync(a.ws.tested + a.rows, 0, sizeof(int32_t), stream);
+    if (err != cudaSuccess) return err;
+    const int64_t nwin = a.rows / a.window;
+    verify_plan_kernel<<<(unsigned)((nwin + kPlanThreads - 1) / kPlanThreads), kPlanThreads, 0, stream>>>(a);
     count_launch();
-    cudaError_t err = cudaGetLastError();
+    err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     const int nvec = a.n / Elem<T>::kVec;
     const int jv = nvec <= kVThreads ? 1 : (nvec <= 2 * kVThreads ? 2 : (nvec <= 4 * kVThreads ? 4 : 8));
