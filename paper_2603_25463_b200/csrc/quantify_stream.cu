@@ -44,7 +44,7 @@ struct DirectConst {
 
 constexpr int kPark = 16;      // rows parked before the CTA finishes them, one per warp
 constexpr int kListCap = 704;  // > 256 e for r <= 1: more codes than that cannot exceed theta
-constexpr int kParkList = 48;  // listed codes a parked row can carry; a longer list is finished at once
+constexpr int kParkList = 32;  // listed codes a parked row carries itself; the rest of a longer list sits in a shared buffer
 
 // A row whose sweeps are done and whose arithmetic is still to do.
 struct Parked {
@@ -55,6 +55,7 @@ struct Parked {
     float c0, th;  // series route: centre of the power sums and clamp level, in units of exp(c - m)
     float rho, r;  // radius as stored, and clamped (after Softplus when raw) as the sweeps used it
     int argmin, nmax, nlist, status, series;
+    int par;  // which of the two shared list buffers holds the codes beyond kParkList
 };
 
 struct QShared {
@@ -65,7 +66,7 @@ struct QShared {
     int bad_nan, bad_finite;
     int abort;
     int nlist;  // codes above theta in the row being swept
-    float list[kListCap];
+    float list[2][kListCap];  // by row parity: a long list must outlive the next row's sweeps
     Parked park[kPark];
 };
 static_assert(sizeof(QShared) + kQStages * 32768 <= 115712, "two CTAs per SM must fit in shared memory");
@@ -141,7 +142,7 @@ __device__ __noinline__ void finish_row(const QuantifyArgs &a, const Parked &pk,
     const ciar_quantify_out &o = a.out;
     const long long lr = pk.lr;
     if (pk.status) {
-        if (lane == 0 && pk.status > 0) write_unusable(o, lr, pk.status);  // negative: finished earlier
+        if (lane == 0) write_unusable(o, lr, pk.status);
         return;
     }
     const bool series = pk.series != 0;
@@ -332,23 +333,20 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
         if (lr < a.rows && map_row(a.rm, lr, pr)) return reinterpret_cast<const float *>(a.radius)[pr];
         return 0.f;
     };
-    // a row whose list outgrew its slot: the slot's part joins the rest in the CTA's list (one warp)
-    auto finish_long = [&](Parked &p) {
-        for (int i = lane; i < kParkList; i += 32) sh.list[i] = p.list[i];
-        __syncwarp();
-        finish_row(a, p, sh.list, lane);
-        __syncwarp();
-        if (lane == 0) p.status = -1;  // done
-    };
-    // every warp finishes one parked row
+    // Every warp finishes one parked row.  A row whose list outgrew its slot first moves the slot's
+    // part next to the rest, which waits in the shared buffer of the row's parity.
     auto finish_parked = [&](int count) {
         __syncthreads();
         if (warp < count) {
             Parked &p = sh.park[warp];
-            if (p.status >= 0) {
-                if (p.nlist > kParkList) finish_long(p);
-                else finish_row(a, p, p.list, lane);
+            const float *list = p.list;
+            if (p.nlist > kParkList) {
+                float *big = sh.list[p.par];
+                for (int i = lane; i < kParkList; i += 32) big[i] = p.list[i];
+                __syncwarp();
+                list = big;
             }
+            finish_row(a, p, list, lane);
         }
         __syncthreads();
     };
@@ -360,6 +358,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
 
     uint32_t phases = 0;
     int k = 0, filled = 0;
+    int par = 0;  // alternates with every row swept: which shared list buffer the row's long list uses
     bool aborted = false;
     for (;; ++k) {
         const int64_t lr = blockIdx.x + (int64_t)k * stride_rows;
@@ -400,12 +399,9 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             aborted = true;
             break;
         }
-        if (filled > 0 && sh.park[filled - 1].nlist > kParkList && sh.park[filled - 1].status >= 0) {
-            // the row parked last listed more codes than its slot holds; the rest sits in the CTA's
-            // list, which this row is about to reuse: finish that row now
-            if (warp == 0) finish_long(sh.park[filled - 1]);
-            named_bar_sync(kBarRow, kQThreads);
-        }
+        // the row parked last listed more codes than its slot holds: its shared buffer is reused two
+        // rows on, so the parked rows are finished at the end of this row
+        const bool long_pending = filled > 0 && sh.park[filled - 1].nlist > kParkList;
         const float m = warp_redux_max(sh.wmax[lane & (kQWarps - 1)]);
         if (tm == m) {  // this thread holds a maximum: its lowest index competes for the arg-max
             int best = INT_MAX;
@@ -537,7 +533,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
                             if (ev > th) {
                                 const int slot = atomicAdd(&pk.nlist, 1);
                                 if (slot < kParkList) pk.list[slot] = ev;
-                                else if (slot < kListCap) sh.list[slot] = ev;
+                                else if (slot < kListCap) sh.list[par][slot] = ev;
                                 ev = th;
                             }
                         }
@@ -619,8 +615,10 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             pk.nmax = nmax;
             pk.status = status;
             pk.series = series;
+            pk.par = par;
         }
-        if (++filled == kPark) {
+        par ^= 1;
+        if (++filled == kPark || long_pending) {
             finish_parked(filled);
             filled = 0;
         }

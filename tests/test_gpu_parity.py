@@ -107,6 +107,27 @@ def test_quantify_degenerate_rows(ciar):
             assert out.argmax.cpu().numpy()[4] == 40
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_quantify_streaming_rows_with_many_large_codes(ciar, dtype):
+    """Rows of the streaming quantifier (>= 2048 codes) in which tens to hundreds of codes sit above
+    the probability level that is treated exactly, several such rows in a row, mixed with ordinary
+    ones, for radii on both sides of 1 (series and direct routes)."""
+    v = 4096
+    g = torch.Generator().manual_seed(123)
+    rows = []
+    for tops in (1, 40, 200, 600, 3, 650, 650, 33, 32, 31, 0, 256):
+        row = torch.randn(v, generator=g) * 0.5 - 6.0
+        idx = torch.randperm(v, generator=g)[:tops]
+        row[idx] = 5.0 + 0.01 * torch.randn(tops, generator=g)
+        rows.append(row)
+    logits = torch.stack(rows * 3).to(dtype)  # 36 rows: more than one batch of parked rows
+    n = logits.shape[0]
+    radius = torch.tensor([0.05, 1.0, 0.3, 0.9, 2.5, 1.0] * (n // 6))
+    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=radius, tau=1e-3)
+    ref, out, rep = pu.check_quantify(logits, prm)
+    assert rep.near_tie_flags <= 1
+
+
 def test_quantify_policies(ciar):
     rows, v = 64, 1024
     logits = _logits(rows, v, torch.bfloat16, scale=2.0, seed=21)
