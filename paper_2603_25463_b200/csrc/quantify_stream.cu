@@ -186,44 +186,48 @@ __device__ __noinline__ void finish_row(const QuantifyArgs &a, const Parked &pk,
 #pragma unroll
             for (int q = 0; q < 6; ++q) ls[q] = warp_sum_d(ls[q]);
         }
-        const double nl = (double)nlist;
+        // Unlisted codes enter through G_k = sum of (x - x0)^k: the power sums over all codes (listed ones
+        // clamped to theta) less the clamped codes' share.
+        const double nl = (double)nlist, nu = nn - nl;
         const double x0 = c0 * invz, hth = (th - c0) * invz;
-        const double iz2 = invz * invz;
-        const double H1 = (zd - ls[0] - nn * c0) * invz;  // sum of (clamped x - x0)
-        const double H2 = v[2] * iz2, H3 = v[3] * iz2 * invz, H4 = v[4] * iz2 * iz2;
-        // Taylor coefficients about x0 of p^l(x) = x / (b - beta x) and p^u(x) = b x / (1 + beta x)
-        const double u = b - beta * x0, w = 1.0 + beta * x0;
-        const double iuw = fast_rcp(u * w), iu = w * iuw, iw = u * iuw;
-        const double rl = beta * iu, ru = -beta * iw;
-        const double PL0 = x0 * iu, PL1 = b * iu * iu, PL2 = PL1 * rl, PL3 = PL2 * rl, PL4 = PL3 * rl;
-        const double PU1 = b * iw * iw, PU2 = PU1 * ru, PU3 = PU2 * ru, PU4 = PU3 * ru;
-        const double DD0 = kap * x0 * (1.0 - x0) * iuw;                        // p^u - p^l at x0, no cancellation
-        const double DD1 = b * beta * (1.0 - 2.0 * x0) * (u + w) * iuw * iuw;  // PU1 - PL1, no cancellation
-        const double DD2 = PU2 - PL2, DD3 = PU3 - PL3, DD4 = PU4 - PL4;
-        const double h2 = hth * hth, h3 = h2 * hth, h4 = h2 * h2;
-        // what a code clamped to theta contributed through the power sums
-        const double pl_th = PL0 + PL1 * hth + PL2 * h2 + PL3 * h3 + PL4 * h4;
-        const double dd_th = DD0 + DD1 * hth + DD2 * h2 + DD3 * h3 + DD4 * h4;
-        const double B = nn * PL0 + PL1 * H1 + PL2 * H2 + PL3 * H3 + PL4 * H4 + (ls[1] - nl * pl_th);  // sum of raw p^l
-        const double A = nn * DD0 + DD1 * H1 + DD2 * H2 + DD3 * H3 + DD4 * H4 + (ls[2] - nl * dd_th);  // sum of raw widths
+        const double iz2 = invz * invz, h2 = hth * hth;
+        const double G1 = (zd - ls[0] - nn * c0) * invz - nl * hth;
+        const double G2 = v[2] * iz2 - nl * h2, G3 = v[3] * iz2 * invz - nl * h2 * hth, G4 = v[4] * iz2 * iz2 - nl * h2 * h2;
+        // Taylor coefficients about x0 of p^l(x) = x / (b - beta x) and of d(x) = p^u - p^l, p^u(x) = b x / (1 + beta x),
+        // and what the sums need of them (they do not outlive this block)
+        double PL0, DD0, Bd, Ad, Qdd, Qdp, Qpp;
+        {
+            const double u = b - beta * x0, w = 1.0 + beta * x0;
+            const double iuw = fast_rcp(u * w), iu = w * iuw, iw = u * iuw;
+            const double rl = beta * iu, ru = -beta * iw;
+            PL0 = x0 * iu;
+            DD0 = kap * x0 * (1.0 - x0) * iuw;  // p^u - p^l at x0, no cancellation
+            const double PL1 = b * iu * iu, PL2 = PL1 * rl, PL3 = PL2 * rl, PL4 = PL3 * rl;
+            const double PU2 = b * iw * iw * ru, PU3 = PU2 * ru, PU4 = PU3 * ru;
+            const double DD1 = b * beta * (1.0 - 2.0 * x0) * (u + w) * iuw * iuw;  // PU1 - PL1, no cancellation
+            const double DD2 = PU2 - PL2, DD3 = PU3 - PL3, DD4 = PU4 - PL4;
+            Bd = PL1 * G1 + PL2 * G2 + PL3 * G3 + PL4 * G4;
+            Ad = DD1 * G1 + DD2 * G2 + DD3 * G3 + DD4 * G4;
+            // sums of products of the first-order-and-up parts, to fourth order
+            Qpp = PL1 * PL1 * G2 + 2.0 * PL1 * PL2 * G3 + (2.0 * PL1 * PL3 + PL2 * PL2) * G4;
+            Qdd = DD1 * DD1 * G2 + 2.0 * DD1 * DD2 * G3 + (2.0 * DD1 * DD3 + DD2 * DD2) * G4;
+            Qdp = DD1 * PL1 * G2 + (DD1 * PL2 + DD2 * PL1) * G3 + (DD1 * PL3 + DD3 * PL1 + DD2 * PL2) * G4;
+        }
+        const double B = nu * PL0 + Bd + ls[1];  // sum of raw p^l
+        const double A = nu * DD0 + Ad + ls[2];  // sum of raw widths
         S_lo = B;
         S_up = A + B;
         const double rs = S_lo > 0.0 && S_up > 0.0 ? fast_rcp(S_lo * S_up) : 0.0;
         double k_lo = (double)a.lo_cap * S_up * rs, k_up = (double)a.hi_cap * S_lo * rs;
         if (!(S_lo > 0.0) || !(k_lo < 1.0)) k_lo = 1.0;
         if (!(S_up > 0.0) || !(k_up > 1.0)) k_up = 1.0;
-        const double g = k_up - k_lo;  // delta = k_up (p^u - p^l) + g p^l
+        const double g = k_up - k_lo;  // delta = k_up d + g p^l
         omega = k_up * A + g * B;
         const double mu = omega * inv_nn;
-        const double E0 = k_up * DD0 + g * PL0 - mu, E1 = k_up * DD1 + g * PL1, E2 = k_up * DD2 + g * PL2,
-                     E3 = k_up * DD3 + g * PL3, E4 = k_up * DD4 + g * PL4;
-        const double q11 = E1 * E1, q12 = 2.0 * E1 * E2, q22 = 2.0 * E1 * E3 + E2 * E2;
-        const double sq_th = E0 * E0 + 2.0 * E0 * (E1 * hth + E2 * h2 + E3 * h3 + E4 * h4) + q11 * h2 + q12 * h3 + q22 * h4;
-        // listed codes: sum of (delta - mu)^2 from their five exact sums
-        const double sl = k_up * k_up * ls[5] + 2.0 * k_up * g * ls[4] + g * g * ls[3] - 2.0 * mu * (k_up * ls[2] + g * ls[1]) +
-                          nl * mu * mu;
-        ss = nn * E0 * E0 + 2.0 * E0 * (E1 * H1 + E2 * H2 + E3 * H3 + E4 * H4) + q11 * H2 + q12 * H3 + q22 * H4 +
-             (sl - nl * sq_th);
+        const double E0 = k_up * DD0 + g * PL0 - mu;  // delta - mu at x0
+        // sum of (delta - mu)^2: unlisted codes from the expansion, listed codes from their five exact sums
+        ss = nu * E0 * E0 + 2.0 * E0 * (k_up * Ad + g * Bd) + k_up * k_up * Qdd + 2.0 * k_up * g * Qdp + g * g * Qpp +
+             (k_up * k_up * ls[5] + 2.0 * k_up * g * ls[4] + g * g * ls[3] - 2.0 * mu * (k_up * ls[2] + g * ls[1]) + nl * mu * mu);
     } else {
         const DirectConst dc = make_direct_const(pk.r, a.n);  // the same constants as the sweep used
         const double P1 = v[2], D1 = v[3], PP = v[4], PD = v[5], DD = v[6];
