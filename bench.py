@@ -296,6 +296,80 @@ def cpu_oracle_baseline(wl, sample_rows, threads=0):
             "sample": "first %d rows of %s (quantify + verify), %.2f s wall" % (rows, wl.name, dt)}
 
 
+def run_decode(args):
+    """Serving decode loop (--workload decode): `requests` concurrent requests, each generating
+    seq_len tokens in draft windows; one step = ciar_decode_step for every unfinished request.
+    Reports the whole loop's tokens/s and the per-step device latency (CUDA events around each step)."""
+    from paper_2603_25463_b200 import ciar
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local if world > 1 else 0)
+    wl = ciar_dist.rank_workload(synth.WORKLOADS["decode"], rank)
+    if args.decode_requests:
+        wl = wl.scaled(images=args.decode_requests)
+    inp = synth.make_inputs(wl, device=dev)
+    req, seq = wl.images, wl.tokens_per_image
+    params = ciar.IntervalParams(radius_mode=ciar.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
+    state = ciar.DecodeState.allocate(req, seq, dev)
+    ws = ciar.alloc_workspace(req * wl.window, wl.window, dev)
+
+    def loop(record):
+        ciar.decode_init(state, 0)
+        events = []
+        steps = 0
+        while True:
+            if record:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            ciar.decode_step(state, inp.draft, inp.target, inp.tokens, inp.u_accept, inp.u_resample, params, wl.window,
+                             ciar.VERIFY_ANCHORED, ws, wl.valid_begin, wl.n_valid)
+            if record:
+                e1.record()
+                events.append((e0, e1))
+            steps += 1
+            if steps % 16 == 0 and int(state.counters[7].item()) >= req:  # every request has finished
+                break
+            if steps > 4 * seq:
+                raise RuntimeError("decode loop did not finish")
+        return steps, events
+
+    loop(False)  # warm-up: one whole generation
+    torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index or 0)
+    launches0 = ciar.launch_count()
+    sampler.start()
+    barrier(world)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    steps, events = loop(True)
+    t1.record()
+    barrier(world)
+    clocks = sampler.stop()
+    launches = ciar.launch_count() - launches0
+    total_ms = max_over_ranks(t0.elapsed_time(t1), world)
+    cnt = state.counters.cpu().numpy()
+    # steps after the last request finished do no work but are inside the timed region: count only useful ones
+    lat = np.array([a.elapsed_time(b) for a, b in events]) * 1e3
+    useful = int(np.ceil(cnt[0] / req)) if req else 0
+    if rank != 0:
+        return
+    print(json.dumps({
+        "metric": METRIC, "value": world * req * seq / (total_ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
+        "steps": steps, "warmup": 1, "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "decode", "requests_per_gpu": req, "seq_len": seq, "vocab": wl.vocab, "logits": wl.dtype,
+                   "window": wl.window, "verify_mode": "anchored", "radius": "per_row", "tau": wl.tau,
+                   "l2": "pools of %.1f GB, rows touched once" % (2 * req * seq * wl.vocab * wl.elem_bytes / 1e9)},
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "gpu_launches": int(launches),
+        "step_latency_us": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)),
+                            "max": float(lat.max()), "timed_with": "CUDA events around every ciar_decode_step"},
+        "decode": {"windows": int(cnt[0]), "cloud_call_windows": int(cnt[1]), "rows_sent": int(cnt[2]),
+                   "rows_flagged": int(cnt[3]), "draft_tokens_kept": int(cnt[4]), "resampled": int(cnt[5]),
+                   "rows_quantified": int(cnt[6]), "useful_steps": useful},
+    }))
+
+
 def run_reference(args):
     """The base contract's reference arm: here the CPU oracle on host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -342,6 +416,7 @@ def main():
     ap.add_argument("--workload", default="llamagen384", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--cpu-rows", type=int, default=9216, help="rows of the CPU oracle's bounded sample")
+    ap.add_argument("--decode-requests", type=int, default=0, help="decode workload: concurrent requests (default 256)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -351,7 +426,10 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the CIAR path has no CPU fallback "
                          "(use --impl reference for the CPU oracle)")
-    run_ours(args)
+    if args.workload == "decode":
+        run_decode(args)
+    else:
+        run_ours(args)
     if int(os.environ.get("WORLD_SIZE", "1")) > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
