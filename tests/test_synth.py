@@ -74,3 +74,20 @@ def test_gumbel_tokens_follow_the_draft_row():
     expect = (p ** 2).sum(1)  # E[p_x] for x ~ p
     z = (picked - expect).sum() / np.sqrt(((p ** 3).sum(1) - expect ** 2).sum())
     assert abs(z) < 4.5
+
+
+def test_tau_sits_between_the_two_token_classes():
+    """tests/golden/tau_calibration.txt (written from the CPU oracle by the script beside it): the
+    frozen threshold of every workload lies strictly between the highest interior score and the
+    lowest boundary score, so no flag decision of the parity workloads is a near tie."""
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "tau_calibration.txt")
+    seen = set()
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        name, rows, hi_int, lo_bnd, mid, tau, frac = line.split()
+        assert float(hi_int) * 2 < float(tau) < float(lo_bnd) / 2, name
+        assert float(tau) == synth.WORKLOADS[name].tau
+        seen.add(name)
+    assert seen == set(synth.WORKLOADS)
