@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyArgs a)
                 }
 
                 if (!acc) {
-                    cand = resample_row(rd, rt, mp, zp, mq, zq, a.u_resample[pr], a.vb, scan_warp, sh_i + 2);
+                    cand = resample_row<T, kThreads>(rd, rt, mp, zp, mq, zq, a.u_resample[pr], a.vb, scan_warp, sh_i + 2);
                 }
             }
         }

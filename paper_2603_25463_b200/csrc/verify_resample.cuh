@@ -1,4 +1,4 @@
-// Residual resampling of one rejected row by a whole CTA (kThreads threads): the token drawn from
+// Residual resampling of one rejected row by a whole CTA (NT threads): the token drawn from
 // norm(max(0, q - p)) by inverse CDF, p = softmax(draft row), q = softmax(target row).
 #pragma once
 
@@ -17,9 +17,9 @@ __device__ __forceinline__ float residual_term(float t, float c, float mq, float
 // Smallest code k whose cumulative residual exceeds u * total (cumulated in code order); the last
 // code with a positive residual if rounding leaves none; the mode of q (lowest index) when the
 // residual mass is zero.  Returns the global code id.  (mp, zp) / (mq, zq): maximum and sum of
-// exp(. - max) of the draft / target row.  scan_warp: kWarps doubles, sh_i: 2 ints of shared
+// exp(. - max) of the draft / target row.  scan_warp: NT / 32 doubles, sh_i: 2 ints of shared
 // memory.  Every thread of the CTA must call it; all get the result.
-template <typename T>
+template <typename T, int NT>
 __device__ __forceinline__ int32_t resample_row(const RowView<T> &rd, const RowView<T> &rt, float mp, double zp, float mq,
                                                 double zq, float u_res, int32_t vb, double *scan_warp, int *sh_i)
 {
@@ -32,7 +32,7 @@ __device__ __forceinline__ int32_t resample_row(const RowView<T> &rd, const RowV
     // Thread t owns a contiguous run of vectors so that a block scan gives code-order prefixes.
     const float ratio = (float)(zq / zp);
     const int32_t nvec = rt.vec_end - rt.vec_begin;
-    const int32_t vpt = (nvec + kThreads - 1) / kThreads;
+    const int32_t vpt = (nvec + NT - 1) / NT;
     const int32_t v0 = rt.vec_begin + threadIdx.x * vpt;
     const int32_t v1 = min(v0 + vpt, rt.vec_end);
     double part = 0.0;
@@ -56,7 +56,7 @@ __device__ __forceinline__ int32_t resample_row(const RowView<T> &rd, const RowV
     __syncthreads();
     double woff = 0.0, total = 0.0;
 #pragma unroll
-    for (int ww = 0; ww < kWarps; ++ww) {
+    for (int ww = 0; ww < NT / 32; ++ww) {
         if (ww < warp) woff += scan_warp[ww];
         total += scan_warp[ww];
     }
@@ -106,7 +106,7 @@ __device__ __forceinline__ int32_t resample_row(const RowView<T> &rd, const RowV
     } else {
         // p == q wherever q > 0: fall back to the mode of q (lowest index at the maximum)
         int32_t amin = 0x7fffffff;
-        for (int32_t vi = rt.vec_begin + threadIdx.x; vi < rt.vec_end; vi += kThreads) {
+        for (int32_t vi = rt.vec_begin + threadIdx.x; vi < rt.vec_end; vi += NT) {
             float tv[V];
             const int32_t i0 = rt.load(vi, tv, -INFINITY);
 #pragma unroll

@@ -21,6 +21,7 @@ constexpr int kVWarps = kVThreads / 32;
 constexpr int kVStages = 3;
 constexpr int kVPark = 16;
 constexpr int kPlanThreads = 128;
+constexpr int kWinThreads = 512;  // threads that resample one rejected window
 constexpr long long kWaitCycles = 2000000000ll;
 constexpr long long kDrainCycles = 20000000ll;
 
@@ -327,9 +328,9 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
 
 // ---- window: accepted length and, for a rejected window, the residual sample of its first rejected row
 template <typename T>
-__global__ void __launch_bounds__(kThreads) verify_window_kernel(VerifyArgs a)
+__global__ void __launch_bounds__(kWinThreads) verify_window_kernel(VerifyArgs a)
 {
-    __shared__ double scan_warp[kWarps];
+    __shared__ double scan_warp[kWinThreads / 32];
     __shared__ int sh_i[2];
     __shared__ int sh_a;
     const T *dbase = reinterpret_cast<const T *>(a.draft);
@@ -367,7 +368,7 @@ __global__ void __launch_bounds__(kThreads) verify_window_kernel(VerifyArgs a)
             if (zq > 0.0 && zq < INFINITY && zp > 0.0 && zp < INFINITY && mp == mp) {
                 const RowView<T> rd(dbase + pr * a.row_stride, a.vb, a.n);
                 const RowView<T> rt(tbase + pr * a.row_stride, a.vb, a.n);
-                tok = resample_row(rd, rt, mp, zp, mq, zq, a.u_resample[pr], a.vb, scan_warp, sh_i);
+                tok = resample_row<T, kWinThreads>(rd, rt, mp, zp, mq, zq, a.u_resample[pr], a.vb, scan_warp, sh_i);
             }
         }
         if (threadIdx.x == 0) {
@@ -422,9 +423,9 @@ cudaError_t launch_all(const VerifyArgs &a, cudaStream_t stream)
     }
     if (err != cudaSuccess) return err;
     const int64_t nw = a.rows / a.window;
-    const int64_t cap = (int64_t)sm_count() * 8;
+    const int64_t cap = (int64_t)sm_count() * 4;
     const unsigned grid = (unsigned)(nw < cap ? nw : cap);
-    verify_window_kernel<T><<<grid, kThreads, 0, stream>>>(a);
+    verify_window_kernel<T><<<grid, kWinThreads, 0, stream>>>(a);
     count_launch();
     return cudaGetLastError();
 }
