@@ -403,9 +403,6 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             aborted = true;
             break;
         }
-        // the row parked last listed more codes than its slot holds: its shared buffer is reused two
-        // rows on, so the parked rows are finished at the end of this row
-        const bool long_pending = filled > 0 && sh.park[filled - 1].nlist > kParkList;
         const float m = warp_redux_max(sh.wmax[lane & (kQWarps - 1)]);
         if (tm == m) {  // this thread holds a maximum: its lowest index competes for the arg-max
             int best = INT_MAX;
@@ -473,8 +470,15 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             zs = zz;
             atomicAdd(&sh.nmax, cnt);
         }
-        const float zt = warp_sum_pair(zs, ts, lane);  // lanes 0..15: z, lanes 16..31: t
-        if (lane == 0) sh.wz[warp] = zt;
+        Parked &pk = sh.park[filled];
+        {
+            const float zt = warp_sum_pair(zs, ts, lane);  // lanes 0..15: z, lanes 16..31: t
+            if (lane == 0) {
+                sh.wz[warp] = zt;
+                pk.wsum[warp][0] = zt;
+            }
+            if (lane == 16) pk.wsum[warp][1] = zt;
+        }
         __syncwarp();
         named_bar_sync(kBarRow, kQThreads);
         float z = sh.wz[lane & (kQWarps - 1)];
@@ -514,8 +518,6 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             fence_proxy_async_smem();
             issue(k + kQStages);
         }
-        Parked &pk = sh.park[filled];
-
         // ---- sweep 3: interval sums
         const float c0 = z * inv_n, th = 0.00390625f * ex2_approx(-r * kLog2e) * z;  // clamp level: theta = 2^-8 e^-r
         float r0 = 0.f, r1 = 0.f, r2 = 0.f;  // warp sums: r0, r1 hold two sums each (lanes 0..15 / 16..31)
@@ -596,13 +598,11 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
 
         // ---- park the row's sums
         if (lane == 0) {
-            pk.wsum[warp][0] = zt;
             pk.wsum[warp][2] = r0;
             pk.wsum[warp][4] = r1;
             pk.wsum[warp][6] = r2;
         }
         if (lane == 16) {
-            pk.wsum[warp][1] = zt;
             pk.wsum[warp][3] = r0;
             if (direct) pk.wsum[warp][5] = r1;
         }
@@ -622,6 +622,9 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             pk.par = par;
         }
         par ^= 1;
+        // A row parked before this one may have listed more codes than its slot holds; the rest sits in the
+        // shared buffer of its parity, which the row after this one reuses: finish the parked rows now.
+        const bool long_pending = filled > 0 && sh.park[filled - 1].nlist > kParkList;
         if (++filled == kPark || long_pending) {
             finish_parked(filled);
             filled = 0;
