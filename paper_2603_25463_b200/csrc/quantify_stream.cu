@@ -307,32 +307,32 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
     __syncthreads();
 
     const int nvec = a.n / VEC;
-    const uint32_t row_bytes = (uint32_t)nvec * 16u;
     int nj = JV;
     if (!FULL) {
         nj = (nvec - tid + kQThreads - 1) / kQThreads;
         nj = nj < 0 ? 0 : (nj > JV ? JV : nj);
     }
-    const T *base = reinterpret_cast<const T *>(a.logits) + a.vb;
     const ciar_quantify_out &o = a.out;
-    const int64_t stride_rows = gridDim.x;
-    const float inv_n = 1.0f / (float)a.n;
-    const bool per_row = a.radius_mode == CIAR_RADIUS_PER_ROW;
+    // (row indices, pointers and sizes are formed from the kernel arguments where they are used: nothing
+    // that can be recomputed in an instruction or two is kept in a register across the sweeps)
+    auto row_of = [&](int k) -> int64_t { return blockIdx.x + (int64_t)k * gridDim.x; };
 
     // issues the copy of this CTA's k-th row into its stage (thread 0 only)
     auto issue = [&](int k) {
-        const int64_t lr = blockIdx.x + (int64_t)k * stride_rows;
+        const int64_t lr = row_of(k);
         int64_t pr;
         if (lr < a.rows && map_row(a.rm, lr, pr)) {
             const int s = k % kQStages;
+            const uint32_t row_bytes = (uint32_t)(a.n / VEC) * 16u;
             mbar_arrive_expect_tx(&sh.full[s], row_bytes);
-            bulk_copy_g2s(smem + (size_t)s * kStageBytes, base + pr * a.row_stride, row_bytes, &sh.full[s]);
+            bulk_copy_g2s(smem + (size_t)s * kStageBytes, reinterpret_cast<const T *>(a.logits) + a.vb + pr * a.row_stride,
+                          row_bytes, &sh.full[s]);
         }
     };
     // the stored radius of this CTA's k-th row (every thread reads it, one row ahead of its use)
     auto radius_of = [&](int k) -> float {
-        if (!per_row) return a.r_scalar;
-        const int64_t lr = blockIdx.x + (int64_t)k * stride_rows;
+        if (a.radius_mode != CIAR_RADIUS_PER_ROW) return a.r_scalar;
+        const int64_t lr = row_of(k);
         int64_t pr;
         if (lr < a.rows && map_row(a.rm, lr, pr)) return reinterpret_cast<const float *>(a.radius)[pr];
         return 0.f;
@@ -358,28 +358,27 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
 #pragma unroll
         for (int s = 0; s < kQStages; ++s) issue(s);
     }
-    float rho_next = radius_of(0);
 
     uint32_t phases = 0;
     int k = 0, filled = 0;
     int par = 0;  // alternates with every row swept: which shared list buffer the row's long list uses
     bool aborted = false;
     for (;; ++k) {
-        const int64_t lr = blockIdx.x + (int64_t)k * stride_rows;
-        if (lr >= a.rows) break;
         const int s = k % kQStages;
-        int64_t pr;
-        const bool active = map_row(a.rm, lr, pr);
-        const float rho = rho_next;
-        rho_next = radius_of(k + 1);
-        if (!active) {  // a position past the end of the sequence: nothing to quantify
-            if (tid == 0) {
-                if (o.flag) o.flag[lr] = 0;
-                if (o.row_status) o.row_status[lr] = 0;
-                issue(k + kQStages);
+        {
+            const int64_t lr = row_of(k);
+            if (lr >= a.rows) break;
+            int64_t pr;
+            if (!map_row(a.rm, lr, pr)) {  // a position past the end of the sequence: nothing to quantify
+                if (tid == 0) {
+                    if (o.flag) o.flag[lr] = 0;
+                    if (o.row_status) o.row_status[lr] = 0;
+                    issue(k + kQStages);
+                }
+                continue;
             }
-            continue;
         }
+        const float rho = radius_of(k);  // needed after the second sweep: the load has long landed by then
         const unsigned char *stage = smem + (size_t)s * kStageBytes;
         if (mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kWaitCycles)) phases ^= 1u << s;
         else sh.abort = 1;
@@ -519,7 +518,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             issue(k + kQStages);
         }
         // ---- sweep 3: interval sums
-        const float c0 = z * inv_n, th = 0.00390625f * ex2_approx(-r * kLog2e) * z;  // clamp level: theta = 2^-8 e^-r
+        const float c0 = z * rcp_approx((float)a.n), th = 0.00390625f * ex2_approx(-r * kLog2e) * z;  // clamp level: theta = 2^-8 e^-r
         float r0 = 0.f, r1 = 0.f, r2 = 0.f;  // warp sums: r0, r1 hold two sums each (lanes 0..15 / 16..31)
         if (!status && series) {
             // Codes above th are listed and clamped to th.  Most threads hold none (seen from the thread's
@@ -607,6 +606,9 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             if (direct) pk.wsum[warp][5] = r1;
         }
         if (tid == 0) {
+            const int64_t lr = row_of(k);
+            int64_t pr;
+            map_row(a.rm, lr, pr);
             pk.lr = lr;
             pk.pr = pr;
             pk.m = m;
@@ -636,7 +638,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
         // A copy never arrived.  Mark this row and the rest of this CTA's rows, then give the
         // copies still in flight a last bounded chance to land before the CTA leaves.
         for (int k2 = k;; ++k2) {
-            const int64_t lr = blockIdx.x + (int64_t)k2 * stride_rows;
+            const int64_t lr = row_of(k2);
             if (lr >= a.rows) break;
             write_unusable(o, lr, CIAR_ROW_TIMEOUT);
         }
