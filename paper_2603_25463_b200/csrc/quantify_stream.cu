@@ -48,7 +48,9 @@ constexpr int kParkList = 32;  // listed codes a parked row carries itself; the 
 
 // A row whose sweeps are done and whose arithmetic is still to do.
 struct Parked {
-    float wsum[kQWarps][7];  // per-warp sums: 0 exp (terms equal to e0 left out), 1 exp * exponent, 2.. route sums
+    // per-warp sums, as lanes 0 and 16 of each warp hold them: [0] exp (terms equal to e0 left out), [4] exp * exponent,
+    // route sums in [1] [5] [2] [6] [3] (series: powers 2, 3, 4 of e - c0; direct: pl, dd, pl^2, pl dd, dd^2)
+    float wsum[kQWarps][8];
     float list[kParkList];   // series route: exponentials of the codes above theta
     long long lr, pr;
     float m, e0;   // row maximum; the exponential of a code equal to it, as the sweeps computed it
@@ -60,9 +62,9 @@ struct Parked {
 
 struct QShared {
     unsigned long long full[kQStages];
-    float wmax[kQWarps];
-    float wz[kQWarps];
-    int argmin, nmax;  // lowest index holding the row maximum, number of codes whose exponential equals e0
+    // by the row's turn (rows swept so far, low bits): a row's first sweep runs while the row before it is still in use
+    float wmax[2][kQWarps];
+    int argmin[2], nmax[4];  // lowest index holding the row maximum, number of codes whose exponential equals e0
     int bad_nan, bad_finite;
     int abort;
     int nlist;  // codes above theta in the row being swept
@@ -149,9 +151,10 @@ __device__ __noinline__ void finish_row(const QuantifyArgs &a, const Parked &pk,
     double v[7];
 #pragma unroll
     for (int q = 0; q < 7; ++q) {
+        constexpr int kSlot[7] = { 0, 4, 1, 5, 2, 6, 3 };
         v[q] = 0.0;
         if (q < 5 || !series) {
-            if (lane < kQWarps) v[q] = (double)pk.wsum[lane][q];
+            if (lane < kQWarps) v[q] = (double)pk.wsum[lane][kSlot[q]];
             v[q] = warp_sum_d(v[q]);
         }
     }
@@ -329,14 +332,6 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
                           row_bytes, &sh.full[s]);
         }
     };
-    // the stored radius of this CTA's k-th row (every thread reads it, one row ahead of its use)
-    auto radius_of = [&](int k) -> float {
-        if (a.radius_mode != CIAR_RADIUS_PER_ROW) return a.r_scalar;
-        const int64_t lr = row_of(k);
-        int64_t pr;
-        if (lr < a.rows && map_row(a.rm, lr, pr)) return reinterpret_cast<const float *>(a.radius)[pr];
-        return 0.f;
-    };
     // Every warp finishes one parked row.  A row whose list outgrew its slot first moves the slot's
     // part next to the rest, which waits in the shared buffer of the row's parity.
     auto finish_parked = [&](int count) {
@@ -360,59 +355,71 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
     }
 
     uint32_t phases = 0;
-    int k = 0, filled = 0;
-    int par = 0;  // alternates with every row swept: which shared list buffer the row's long list uses
+    int filled = 0;
+    int it = 0;  // rows swept so far: its low bits pick the slot of everything that is double-buffered by row
     bool aborted = false;
-    for (;; ++k) {
-        const int s = k % kQStages;
-        {
-            const int64_t lr = row_of(k);
-            if (lr >= a.rows) break;
+
+    // The next row at or after `from` that has something to quantify (-1: none left).  Positions past
+    // the end of a sequence get their outputs here and hand their stage's turn to a later row.
+    const int nk = (int)((a.rows - blockIdx.x + gridDim.x - 1) / gridDim.x);  // rows this CTA walks (the grid never exceeds the rows)
+    auto next_active = [&](int from) -> int {
+        if (a.rm.pos == nullptr) return from < nk ? from : -1;
+        for (int kk = from;; ++kk) {
+            if (kk >= nk) return -1;
+            const int64_t lr = row_of(kk);
             int64_t pr;
-            if (!map_row(a.rm, lr, pr)) {  // a position past the end of the sequence: nothing to quantify
-                if (tid == 0) {
-                    if (o.flag) o.flag[lr] = 0;
-                    if (o.row_status) o.row_status[lr] = 0;
-                    issue(k + kQStages);
-                }
-                continue;
+            if (map_row(a.rm, lr, pr)) return kk;
+            if (tid == 0) {
+                if (o.flag) o.flag[lr] = 0;
+                if (o.row_status) o.row_status[lr] = 0;
+                issue(kk + kQStages);
             }
         }
-        const float rho = radius_of(k);  // needed after the second sweep: the load has long landed by then
+    };
+    // Waits for row kk to land and takes the maximum over it (sweep 1): each warp's maximum goes to the slot
+    // of the row's turn, and only that is kept.  Thread 0 also clears the row's arg-max and maximum-count slots.
+    auto first_sweep = [&](int kk, int turn) {
+        const int s = kk % kQStages;
         const unsigned char *stage = smem + (size_t)s * kStageBytes;
         if (mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kWaitCycles)) phases ^= 1u << s;
         else sh.abort = 1;
-
-        // ---- sweep 1: the row's maximum
         typename V::Max mx = V::max_init();
 #pragma unroll
         for (int j = 0; j < JV; ++j)
             if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * kQThreads));
-        const float tm = V::max_value(mx);
-        const float wm = warp_redux_max(tm);
-        if (lane == 0) sh.wmax[warp] = wm;
+        const float wm = warp_redux_max(V::max_value(mx));
+        if (lane == 0) sh.wmax[turn & 1][warp] = wm;
         if (tid == 0) {
-            sh.argmin = INT_MAX;
-            sh.nmax = 0;
-            sh.park[filled].nlist = 0;
+            sh.argmin[turn & 1] = INT_MAX;
+            sh.nmax[turn & 3] = 0;
         }
+    };
+
+    int k = next_active(0);
+    if (k >= 0) {
+        first_sweep(k, 0);
         __syncwarp();
         named_bar_sync(kBarRow, kQThreads);
-        if (sh.abort) {
-            aborted = true;
-            break;
+        if (sh.abort) aborted = true;
+    }
+    while (k >= 0 && !aborted) {
+        const int s = k % kQStages;
+        const int par = it & 1;
+        const unsigned char *stage = smem + (size_t)s * kStageBytes;
+        Parked &pk = sh.park[filled];
+        if (tid == 0) {  // the row's place and stored radius: the others read the radius after the barrier
+            const int64_t lr = row_of(k);
+            int64_t pr;
+            map_row(a.rm, lr, pr);
+            pk.nlist = 0;
+            pk.lr = lr;
+            pk.pr = pr;
+            pk.rho = a.radius_mode == CIAR_RADIUS_PER_ROW ? reinterpret_cast<const float *>(a.radius)[pr] : a.r_scalar;
         }
-        const float m = warp_redux_max(sh.wmax[lane & (kQWarps - 1)]);
-        if (tm == m) {  // this thread holds a maximum: its lowest index competes for the arg-max
-            int best = INT_MAX;
-            for (int j = nj - 1; j >= 0; --j) {
-                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
-#pragma unroll
-                for (int q = VEC - 1; q >= 0; --q)
-                    if (Elem<T>::widen(v[q]) == m) best = (tid + j * kQThreads) * VEC + q;
-            }
-            if (best != INT_MAX) atomicMin(&sh.argmin, best);
-        }
+        const float m = warp_redux_max(sh.wmax[par][lane & (kQWarps - 1)]);
+        // ---- sweep 1 of the row after this one, so that one barrier per row serves both
+        const int kn = next_active(k + 1);
+        if (kn >= 0) first_sweep(kn, it + 1);
 
         // ---- sweep 2: exponentials (kept in registers), their sum and the entropy sum
         const float m2 = m * kLog2e;
@@ -428,7 +435,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
 #pragma unroll
                     for (int q = 0; q < NPV; ++q) {
                         const float2 d = __ffma2_rn(c[q], L2, nm2);
-                        const float2 ev = make_float2(ex2_approx(d.x), ex2_approx(d.y));  // a NaN logit poisons the sums on purpose
+                        const float2 ev = make_float2(ex2_once(d.x), ex2_once(d.y));  // a NaN logit poisons the sums on purpose
                         z2 = __fadd2_rn(z2, ev);
                         t2 = __ffma2_rn(ev, d, t2);  // 0 * -inf = NaN for a -inf logit: redone below
                         e[j * NPV + q] = ev;
@@ -454,9 +461,9 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             }
         }
         const float e0 = ex2_approx(fmaf(m, kLog2e, -m2));  // the exponential every maximum got
-        if (tm == m) {
-            // This thread owns a maximum.  A term near 1 would cost the small terms their low bits, so its
-            // partial sum is formed again without the terms equal to e0; they come back exactly, as a count.
+        if (sh.wmax[par][warp] == m) {
+            // This warp owns a maximum.  A term near 1 would cost the small terms their low bits, so its threads
+            // form their partial sums again without the terms equal to e0; they come back exactly, as a count.
             float zz = 0.f;
             int cnt = 0;
 #pragma unroll
@@ -467,24 +474,35 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
                 }
             }
             zs = zz;
-            atomicAdd(&sh.nmax, cnt);
+            if (cnt > 0) {
+                atomicAdd(&sh.nmax[it & 3], cnt);
+                // the thread's lowest index holding the maximum competes for the arg-max
+                int best = INT_MAX;
+                for (int j = nj - 1; j >= 0; --j) {
+                    const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+#pragma unroll
+                    for (int q = VEC - 1; q >= 0; --q)
+                        if (Elem<T>::widen(v[q]) == m) best = (tid + j * kQThreads) * VEC + q;
+                }
+                if (best != INT_MAX) atomicMin(&sh.argmin[par], best);
+            }
         }
-        Parked &pk = sh.park[filled];
         {
             const float zt = warp_sum_pair(zs, ts, lane);  // lanes 0..15: z, lanes 16..31: t
-            if (lane == 0) {
-                sh.wz[warp] = zt;
-                pk.wsum[warp][0] = zt;
-            }
-            if (lane == 16) pk.wsum[warp][1] = zt;
+            if ((lane & 15) == 0) pk.wsum[warp][lane >> 2] = zt;
         }
         __syncwarp();
         named_bar_sync(kBarRow, kQThreads);
-        float z = sh.wz[lane & (kQWarps - 1)];
+        if (sh.abort) {
+            aborted = true;
+            break;
+        }
+        float z = pk.wsum[lane & (kQWarps - 1)][0];
 #pragma unroll
         for (int ofs = 8; ofs > 0; ofs >>= 1) z += __shfl_xor_sync(0xffffffffu, z, ofs);
-        const int nmax = sh.nmax;
+        const int nmax = sh.nmax[it & 3];
         z = fmaf((float)nmax, e0, z);
+        const float rho = pk.rho;
 
         int status = 0;
         if (!(m > -INFINITY) || !(z > 0.f) || !(z < INFINITY)) {
@@ -513,19 +531,32 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
         const float r = row_radius(rho, a.radius_is_raw, a.r_max);
         const bool series = r <= 1.0f;
         const bool direct = !status && !series;
-        if (tid == 0 && !direct) {  // every thread has read the stage: refill it
-            fence_proxy_async_smem();
-            issue(k + kQStages);
+        const float c0 = z * rcp_approx((float)a.n), th = 0.00390625f * ex2_approx(-r * kLog2e) * z;  // clamp level: theta = 2^-8 e^-r
+        if (tid == 0) {
+            if (!direct) {  // every thread has read the stage: refill it
+                fence_proxy_async_smem();
+                issue(k + kQStages);
+            }
+            // the row's scalars, parked as soon as they exist
+            pk.m = m;
+            pk.e0 = e0;
+            pk.c0 = c0;
+            pk.th = th;
+            pk.r = r;
+            pk.argmin = sh.argmin[par];
+            pk.nmax = nmax;
+            pk.status = status;
+            pk.series = series;
+            pk.par = par;
         }
         // ---- sweep 3: interval sums
-        const float c0 = z * rcp_approx((float)a.n), th = 0.00390625f * ex2_approx(-r * kLog2e) * z;  // clamp level: theta = 2^-8 e^-r
         float r0 = 0.f, r1 = 0.f, r2 = 0.f;  // warp sums: r0, r1 hold two sums each (lanes 0..15 / 16..31)
         if (!status && series) {
-            // Codes above th are listed and clamped to th.  Most threads hold none (seen from the thread's
-            // maximum logit), and a vector holding none is skipped on one comparison of its maximum.
-            // (th_log is a slightly low stand-in for log2(th), so the test on the thread's maximum errs on the safe side)
+            // Codes above th are listed and clamped to th.  Most warps hold none (seen from the warp's maximum
+            // logit), and a vector holding none is skipped on one comparison of its maximum.
+            // (th_log is a slightly low stand-in for log2(th), so the test on the warp's maximum errs on the safe side)
             const float th_log = __log2f(th) - 1e-3f;
-            if (__builtin_expect(fmaf(tm, kLog2e, -m2) > th_log, 0)) {
+            if (__builtin_expect(fmaf(sh.wmax[par][warp], kLog2e, -m2) > th_log, 0)) {  // warps whose maximum is below theta hold no such code
 #pragma unroll
                 for (int j = 0; j < JV; ++j) {
                     float2 g = e[j * NPV];
@@ -596,34 +627,12 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
         }
 
         // ---- park the row's sums
-        if (lane == 0) {
-            pk.wsum[warp][2] = r0;
-            pk.wsum[warp][4] = r1;
-            pk.wsum[warp][6] = r2;
+        if ((lane & 15) == 0) {
+            float *w = &pk.wsum[warp][lane >> 2];
+            w[1] = r0;
+            w[2] = r1;
+            w[3] = r2;
         }
-        if (lane == 16) {
-            pk.wsum[warp][3] = r0;
-            if (direct) pk.wsum[warp][5] = r1;
-        }
-        if (tid == 0) {
-            const int64_t lr = row_of(k);
-            int64_t pr;
-            map_row(a.rm, lr, pr);
-            pk.lr = lr;
-            pk.pr = pr;
-            pk.m = m;
-            pk.e0 = e0;
-            pk.c0 = c0;
-            pk.th = th;
-            pk.rho = rho;
-            pk.r = r;
-            pk.argmin = sh.argmin;
-            pk.nmax = nmax;
-            pk.status = status;
-            pk.series = series;
-            pk.par = par;
-        }
-        par ^= 1;
         // A row parked before this one may have listed more codes than its slot holds; the rest sits in the
         // shared buffer of its parity, which the row after this one reuses: finish the parked rows now.
         const bool long_pending = filled > 0 && sh.park[filled - 1].nlist > kParkList;
@@ -631,6 +640,8 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             finish_parked(filled);
             filled = 0;
         }
+        k = kn;
+        ++it;
     }
     if (filled > 0) finish_parked(filled);
 

@@ -107,6 +107,15 @@ __device__ __forceinline__ float warp_sum_pair(float a, float b, int lane)
     return keep;
 }
 
+// 2^x evaluated exactly once, where it is written: the compiler may neither drop nor repeat it, so the
+// result is held rather than formed again from its operand later on.
+__device__ __forceinline__ float ex2_once(float x)
+{
+    float y;
+    asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ float2 f2(float x, float y) { return make_float2(x, y); }
 __device__ __forceinline__ float2 f2(float x) { return make_float2(x, x); }
 
