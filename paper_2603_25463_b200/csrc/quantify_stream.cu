@@ -287,8 +287,9 @@ __device__ __noinline__ void finish_row(const QuantifyArgs &a, const Parked &pk,
     if (o.row_status) o.row_status[lr] = 0;
 }
 
-// FULL: every thread owns exactly JV vectors (the row has 512 * JV of them).
-template <typename T, int JV, int MINB, bool FULL>
+// FULL: every thread owns exactly JV vectors (the row has 512 * JV of them).  MAPPED: the rows go through a
+// position map (decode mode), so some of them hold nothing to quantify.
+template <typename T, int JV, int MINB, bool FULL, bool MAPPED>
 __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const __grid_constant__ QuantifyArgs a)
 {
     typedef Vec<T> V;
@@ -359,21 +360,25 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
     int it = 0;  // rows swept so far: its low bits pick the slot of everything that is double-buffered by row
     bool aborted = false;
 
-    // The next row at or after `from` that has something to quantify (-1: none left).  Positions past
-    // the end of a sequence get their outputs here and hand their stage's turn to a later row.
     const int nk = (int)((a.rows - blockIdx.x + gridDim.x - 1) / gridDim.x);  // rows this CTA walks (the grid never exceeds the rows)
+    // The next row at or after `from` that has something to quantify (-1: none left).
     auto next_active = [&](int from) -> int {
-        if (a.rm.pos == nullptr) return from < nk ? from : -1;
-        for (int kk = from;; ++kk) {
-            if (kk >= nk) return -1;
-            const int64_t lr = row_of(kk);
+        if (!MAPPED) return from < nk ? from : -1;
+        for (int kk = from; kk < nk; ++kk) {
             int64_t pr;
-            if (map_row(a.rm, lr, pr)) return kk;
-            if (tid == 0) {
-                if (o.flag) o.flag[lr] = 0;
-                if (o.row_status) o.row_status[lr] = 0;
-                issue(kk + kQStages);
-            }
+            if (map_row(a.rm, row_of(kk), pr)) return kk;
+        }
+        return -1;
+    };
+    // Thread 0: the positions past the end of a sequence among rows [from, to) get their outputs, and each hands
+    // its stage's turn to the row three further on.  Only called when the stages of those rows are free.
+    auto retire_skipped = [&](int from, int to) {
+        if (!MAPPED) return;
+        for (int kk = from; kk < (to < 0 ? nk : to); ++kk) {
+            const int64_t lr = row_of(kk);
+            if (o.flag) o.flag[lr] = 0;
+            if (o.row_status) o.row_status[lr] = 0;
+            issue(kk + kQStages);
         }
     };
     // Waits for row kk to land and takes the maximum over it (sweep 1): each warp's maximum goes to the slot
@@ -396,6 +401,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
     };
 
     int k = next_active(0);
+    if (tid == 0) retire_skipped(0, k);
     if (k >= 0) {
         first_sweep(k, 0);
         __syncwarp();
@@ -418,8 +424,10 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
         }
         const float m = warp_redux_max(sh.wmax[par][lane & (kQWarps - 1)]);
         // ---- sweep 1 of the row after this one, so that one barrier per row serves both
+        // (a row three or more further on has not been asked for yet: its sweep waits until this row is done)
         const int kn = next_active(k + 1);
-        if (kn >= 0) first_sweep(kn, it + 1);
+        const bool ahead = kn >= 0 && (!MAPPED || kn - k < kQStages);
+        if (ahead) first_sweep(kn, it + 1);
 
         // ---- sweep 2: exponentials (kept in registers), their sum and the entropy sum
         const float m2 = m * kLog2e;
@@ -536,6 +544,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             if (!direct) {  // every thread has read the stage: refill it
                 fence_proxy_async_smem();
                 issue(k + kQStages);
+                retire_skipped(k + 1, kn);
             }
             // the row's scalars, parked as soon as they exist
             pk.m = m;
@@ -623,6 +632,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             if (tid == 0) {
                 fence_proxy_async_smem();
                 issue(k + kQStages);
+                retire_skipped(k + 1, kn);
             }
         }
 
@@ -642,6 +652,12 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
         }
         k = kn;
         ++it;
+        if (MAPPED && k >= 0 && !ahead) {  // the next row's first sweep could not run ahead: it runs here, with a barrier of its own
+            first_sweep(k, it);
+            __syncwarp();
+            named_bar_sync(kBarRow, kQThreads);
+            if (sh.abort) aborted = true;
+        }
     }
     if (filled > 0) finish_parked(filled);
 
@@ -657,7 +673,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
     }
 }
 
-template <typename T, int JV, int MINB, bool FULL>
+template <typename T, int JV, int MINB, bool FULL, bool MAPPED>
 cudaError_t launch_one(const QuantifyArgs &a, cudaStream_t stream)
 {
     constexpr size_t smem = (size_t)kQStages * kQThreads * JV * 16 + sizeof(QShared);
@@ -667,14 +683,14 @@ cudaError_t launch_one(const QuantifyArgs &a, cudaStream_t stream)
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        err = cudaFuncSetAttribute(quantify_stream_kernel<T, JV, MINB, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        err = cudaFuncSetAttribute(quantify_stream_kernel<T, JV, MINB, FULL, MAPPED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)smem);
         if (err != cudaSuccess) return err;
         configured[dev] = true;
     }
     const int64_t cap = (int64_t)sm_count() * MINB;
     const unsigned grid = (unsigned)(a.rows < cap ? a.rows : cap);
-    quantify_stream_kernel<T, JV, MINB, FULL><<<grid, kQThreads, smem, stream>>>(a);
+    quantify_stream_kernel<T, JV, MINB, FULL, MAPPED><<<grid, kQThreads, smem, stream>>>(a);
     count_launch();
     return cudaGetLastError();
 }
@@ -683,8 +699,9 @@ template <typename T, int JV, int MINB>
 cudaError_t launch_jv(const QuantifyArgs &a, cudaStream_t stream)
 {
     const int nvec = a.n / Elem<T>::kVec;
-    if (nvec == kQThreads * JV) return launch_one<T, JV, MINB, true>(a, stream);
-    return launch_one<T, JV, MINB, false>(a, stream);
+    const bool mapped = a.rm.pos != nullptr;
+    if (nvec == kQThreads * JV) return mapped ? launch_one<T, JV, MINB, true, true>(a, stream) : launch_one<T, JV, MINB, true, false>(a, stream);
+    return mapped ? launch_one<T, JV, MINB, false, true>(a, stream) : launch_one<T, JV, MINB, false, false>(a, stream);
 }
 
 }  // namespace

@@ -123,8 +123,8 @@ struct VParked {
 
 struct VShared {
     unsigned long long full[kVStages];
-    float wmax[kVWarps];
-    int nmax, abort;
+    float wmax[2][kVWarps];  // by row parity
+    int nmax[4], abort;       // count of maxima, by row index mod 4
     VParked park[kVPark];
 };
 
@@ -235,29 +235,36 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
     uint32_t phases = 0;
     int k = 0, filled = 0;
     bool aborted = false;
-    for (;; ++k) {
-        const int idx = blockIdx.x + k * stride;
-        if (idx >= total) break;
-        const int s = k % kVStages;
+    // Waits for this CTA's kk-th row to land and takes the maximum over it (sweep 1): each warp's maximum goes
+    // to the slot of the row's parity.  Thread 0 also clears the row's count of maxima.
+    auto first_sweep = [&](int kk) {
+        const int s = kk % kVStages;
         const unsigned char *stage = smem + (size_t)s * kStageBytes;
         if (mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kWaitCycles)) phases ^= 1u << s;
         else sh.abort = 1;
-        // sweep 1: maximum
         typename V::Max mx = V::max_init();
 #pragma unroll
         for (int j = 0; j < JV; ++j)
             if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * kVThreads));
-        const float tm = V::max_value(mx);
-        const float wm = warp_redux_max(tm);
-        if (lane == 0) sh.wmax[warp] = wm;
-        if (tid == 0) sh.nmax = 0;
+        const float wm = warp_redux_max(V::max_value(mx));
+        if (lane == 0) sh.wmax[kk & 1][warp] = wm;
+        if (tid == 0) sh.nmax[kk & 3] = 0;
+    };
+    const int mine = blockIdx.x < total ? (total - 1 - (int)blockIdx.x) / stride + 1 : 0;  // rows this CTA walks
+    if (mine > 0) {
+        first_sweep(0);
         __syncwarp();
         __syncthreads();
-        if (sh.abort) {
-            aborted = true;
-            break;
-        }
-        const float m = warp_redux_max(sh.wmax[lane & (kVWarps - 1)]);
+        if (sh.abort) aborted = true;
+    }
+    // One barrier per row: the maximum sweep of the row after this one runs before it, so the barrier that
+    // completes this row's sum also publishes the next row's maximum.
+    for (; k < mine && !aborted; ++k) {
+        const int s = k % kVStages;
+        const int par = k & 1;
+        const unsigned char *stage = smem + (size_t)s * kStageBytes;
+        const float m = warp_redux_max(sh.wmax[par][lane & (kVWarps - 1)]);
+        if (k + 1 < mine) first_sweep(k + 1);
         // sweep 2: sum of exponentials; terms equal to the maximum's are counted, not summed
         const float m2 = m * kLog2e;
         const float e0 = ex2_approx(fmaf(m, kLog2e, -m2));
@@ -278,7 +285,7 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
             }
         }
         float zs = z2.x + z2.y;
-        if (tm == m) {  // redo this thread's sum without the maxima (kept exactly, as a count)
+        if (sh.wmax[par][warp] == m) {  // a warp holding a maximum redoes its sums without the maxima (kept exactly, as a count)
             float zz = 0.f;
             int cnt = 0;
             for (int j = 0; j < nj; ++j) {
@@ -290,19 +297,23 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
                 }
             }
             zs = zz;
-            atomicAdd(&sh.nmax, cnt);
+            if (cnt > 0) atomicAdd(&sh.nmax[k & 3], cnt);
         }
         const float wz = warp_sum_f(zs);
         VParked &pk = sh.park[filled];
         if (lane == 0) pk.wz[warp] = wz;
-        __syncthreads();  // every thread has read the stage, the count of maxima is complete
+        __syncthreads();  // every thread has read the stage, the count of maxima is complete, the next maximum is out
+        if (sh.abort) {
+            aborted = true;
+            break;
+        }
         if (tid == 0) {
             fence_proxy_async_smem();
             issue(k + kVStages);
-            pk.lr = a.ws.tested[idx];
+            pk.lr = a.ws.tested[blockIdx.x + k * stride];
             pk.m = m;
             pk.e0 = e0;
-            pk.nmax = sh.nmax;
+            pk.nmax = sh.nmax[k & 3];
         }
         if (++filled == kVPark) {
             finish_parked(filled);
@@ -340,18 +351,28 @@ __global__ void __launch_bounds__(kWinThreads) verify_window_kernel(VerifyArgs a
     for (int64_t w = blockIdx.x; w < nw; w += gridDim.x) {
         const int32_t wlen = window_len(a.rm, w);
         const int64_t row0 = w * a.window;
-        if (threadIdx.x == 0) {
+        if (threadIdx.x < 32) {  // the first warp scans the window, a row per lane: the loads go out together
+            const int lane = threadIdx.x;
             int32_t f = 0;
             if (a.mode != CIAR_VERIFY_ALL) {
                 f = wlen;
-                for (int32_t j = 0; j < wlen; ++j)
-                    if (a.flag[row0 + j]) { f = j; break; }
+                for (int32_t base = 0; base < wlen && f == wlen; base += 32) {
+                    const int32_t j = base + lane;
+                    const unsigned mk = __ballot_sync(0xffffffffu, j < wlen && a.flag[row0 + j] != 0);
+                    if (mk) f = base + __ffs((int)mk) - 1;
+                }
             }
             int32_t acc_len = wlen;
-            for (int32_t j = 0; j < wlen; ++j)
-                if (tested_row(a.mode, j, f, wlen, a.flag, row0 + j) && accept_arr[row0 + j] == 0) { acc_len = j; break; }
-            sh_a = acc_len;
-            if (a.out.accepted_len) a.out.accepted_len[w] = acc_len;
+            for (int32_t base = 0; base < wlen && acc_len == wlen; base += 32) {
+                const int32_t j = base + lane;
+                const unsigned mk =
+                    __ballot_sync(0xffffffffu, tested_row(a.mode, j, f, wlen, a.flag, row0 + j) && accept_arr[row0 + j] == 0);
+                if (mk) acc_len = base + __ffs((int)mk) - 1;
+            }
+            if (lane == 0) {
+                sh_a = acc_len;
+                if (a.out.accepted_len) a.out.accepted_len[w] = acc_len;
+            }
         }
         __syncthreads();
         const int32_t acc_len = sh_a;

@@ -381,3 +381,12 @@ def test_decode_workload_shape_few_steps(ciar):
     """The serving workload's per-step shape (V = 16384, window 8) on fewer requests."""
     wl = synth.WORKLOADS["decode"].scaled(images=16, grid_h=8, grid_w=8)
     _decode_compare(ciar, wl)
+
+
+def test_decode_loop_many_requests_finishing_at_different_steps(ciar):
+    """More rows than three per streaming CTA, requests ending at different steps: a CTA's walk then has runs of
+    three and more positions past a sequence end before a live row, whose copy has not been asked for yet."""
+    wl = synth.Workload("dec3", 168, 4, 5, 2048, "bf16", 8, 0.5, seed=15, decode=True, tau=1e-3)  # 1344 rows per step, 20 tokens
+    steps, ost = _decode_compare(ciar, wl)
+    assert steps >= 3 and (ost.pos == wl.tokens_per_image).all()
+
