@@ -128,6 +128,48 @@ def test_quantify_streaming_rows_with_many_large_codes(ciar, dtype):
     assert rep.near_tie_flags <= 1
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("v", [16392, 40000, 65536 + 4096])
+def test_quantify_wide_rows(ciar, v, dtype):
+    """Rows wider than the on-chip kernel takes (two passes, chunk by chunk; the last chunk ragged): ordinary
+    rows of several sharpnesses, many codes above the exactly treated level, the maximum early / late / tied
+    across chunks, -inf stretches longer than a chunk, unusable rows; radii on both sides of 1."""
+    g = torch.Generator().manual_seed(v)
+    rows = []
+    for scale in (8.0, 1.0, 0.01, 3.0):
+        rows.append(torch.randn(v, generator=g) * scale)
+    for tops in (40, 300, 650):
+        row = torch.randn(v, generator=g) * 0.5 - 6.0
+        row[torch.randperm(v, generator=g)[:tops]] = 5.0 + 0.01 * torch.randn(tops, generator=g)
+        rows.append(row)
+    early = torch.randn(v, generator=g); early[5] = 30.0; rows.append(early)
+    late = torch.randn(v, generator=g); late[v - 3] = 30.0; rows.append(late)
+    rising = torch.randn(v, generator=g) + torch.linspace(0.0, 40.0, v); rows.append(rising)  # the running maximum keeps moving
+    ties = torch.zeros(v); ties[[16390, 300, v - 1, 9000]] = 5.0; rows.append(ties)  # arg-max tie across chunks -> lowest index
+    masked = torch.full((v,), float("-inf")); masked[v - 5000:] = torch.randn(5000, generator=g) * 4.0; rows.append(masked)
+    one_hot = torch.full((v,), float("-inf")); one_hot[16388] = 2.5; rows.append(one_hot)
+    rows.append(torch.full((v,), -0.75))  # constant row
+    nan_row = torch.randn(v, generator=g); nan_row[v - 2] = float("nan"); rows.append(nan_row)
+    rows.append(torch.full((v,), float("-inf")))  # no finite code
+    inf_row = torch.randn(v, generator=g); inf_row[20000 % v] = float("inf"); rows.append(inf_row)
+    logits = torch.stack(rows * 2).to(dtype)  # 34 rows: more than one batch of parked rows
+    n = logits.shape[0]
+    radius = torch.tensor(([0.05, 1.0, 0.3, 2.5, 0.9] * n)[:n])
+    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=radius, tau=1e-3)
+    ref, out, rep = pu.check_quantify(logits, prm)
+    st = out.row_status.cpu().numpy()[:17]
+    assert st[14] == oracle.ROW_NAN and st[15] == oracle.ROW_NO_FINITE and st[16] == oracle.ROW_NAN
+    assert out.argmax.cpu().numpy()[10] == 300
+    assert rep.near_tie_flags <= 1
+
+
+def test_quantify_wide_rows_valid_slice(ciar):
+    """A wide valid slice inside a wider row (aligned to 16 bytes), scalar radius."""
+    rows, stride, vb, n = 5, 70000, 1024, 50000
+    logits = _logits(rows, stride, torch.bfloat16, scale=4.0, seed=5)
+    ref, out, rep = pu.check_quantify(logits, oracle.IntervalParams(r_scalar=0.4, tau=1e-4), valid_begin=vb, valid_count=n)
+
+
 def test_quantify_policies(ciar):
     rows, v = 64, 1024
     logits = _logits(rows, v, torch.bfloat16, scale=2.0, seed=21)
