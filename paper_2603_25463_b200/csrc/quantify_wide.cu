@@ -1,8 +1,8 @@
 // Streaming quantifier for rows too wide to sit on chip (more than 16384 codes, scalar or per-row radius).
 //
-// A persistent CTA of 16 warps walks rows blockIdx.x, blockIdx.x + gridDim.x, ...  A row passes twice
-// through the same ring of shared-memory stages as the on-chip kernel uses, 32 KB at a time ("chunks"),
-// filled by bulk (TMA) copies that one thread issues three chunks ahead:
+// One persistent CTA of 32 warps per SM walks rows blockIdx.x, blockIdx.x + gridDim.x, ...  A row passes
+// twice through a ring of three shared-memory stages, 64 KB at a time ("chunks"), filled by bulk (TMA)
+// copies that one thread issues three chunks ahead:
 //   pass A  softmax statistics on line: every warp keeps a running maximum of the codes it has seen and,
 //           per lane, the sums of exp and of exp * exponent relative to it (rescaled when the maximum
 //           moves; codes equal to the maximum are counted, not summed).  The warps' results are joined
@@ -11,24 +11,33 @@
 //           (power sums about Z / n with the few codes above theta listed; or the direct formulas),
 //           accumulated per chunk in float and across chunks in double; the arg-max.
 // A finished row is parked in the same form as the on-chip kernel parks it and finished by the same warp
-// routine.  Each logit is read from HBM twice (north of that only through the L2).
+// routine.  With one CTA per SM the rows in flight (one per SM) stay in the L2 between their two passes, so
+// each logit comes from HBM once; the copies of pass A ask the L2 to keep their lines, those of pass B to
+// drop them.
+#include <type_traits>
+
 #include "quantify_finish.cuh"
 
 namespace ciar {
 
 namespace {
 
+constexpr int kWThreads = 1024;  // one CTA per SM: the rows in flight on the GPU then fit in the L2 between their passes
+constexpr int kWWarps = kWThreads / 32;
+constexpr int kGroups = 2;  // halves of the CTA, each with its own ring and barrier: a row's chunks go to them in turn
+constexpr int kGThreads = kWThreads / kGroups;
 constexpr int kWJ = 4;                       // vectors per thread and chunk
-constexpr int kChunkVecs = kQThreads * kWJ;  // 2048 vectors
+constexpr int kChunkVecs = kGThreads * kWJ;  // 2048 vectors
 constexpr int kChunkBytes = kChunkVecs * 16;
+constexpr int kRingBytes = kQStages * kChunkBytes;
 
 struct WShared {
-    unsigned long long full[kQStages];
+    unsigned long long full[kGroups][kQStages];
     // pass A, per warp: running maximum, sums relative to it, number of codes equal to it, first chunk holding it
-    float wm[kQWarps];
-    double wz[kQWarps], wt[kQWarps];
-    int wcnt[kQWarps], wchunk[kQWarps];
-    double ws[kQWarps][5];  // pass B, per warp: the route's sums
+    float wm[kWWarps];
+    double wz[kWWarps], wt[kWWarps];
+    int wcnt[kWWarps], wchunk[kWWarps];
+    double ws[kWWarps][5];  // pass B, per warp: the route's sums
     // by row parity (a thread may start the next row while another still reads this row's): lowest index holding the
     // maximum, codes above theta so far, what an unusable row contains
     int argmin[2], nlist[2], bad_nan[2], bad_finite[2];
@@ -36,35 +45,39 @@ struct WShared {
     float list[kListCap];  // series route: exponentials of the codes above theta beyond the parked row's own slots
     Parked park[kPark];
 };
-static_assert(sizeof(WShared) + kQStages * kChunkBytes <= 115712, "two CTAs per SM must fit in shared memory");
+static_assert(sizeof(WShared) + kGroups * kRingBytes <= 232448, "the ring and the scratch must fit in one SM's shared memory");
 
-// One step of this CTA's walk: chunk c of pass `pass` (0 = A, 1 = B) of its k-th row.
+// One step of a group's walk: the group's c-th chunk of pass `pass` (0 = A, 1 = B) of the CTA's k-th row.
 struct Item {
     int k, pass, c;
 };
 
 template <typename T>
-__global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __grid_constant__ QuantifyArgs a)
+__global__ void __launch_bounds__(kWThreads, 1) quantify_wide_kernel(const __grid_constant__ QuantifyArgs a)
 {
     typedef Vec<T> V;
     constexpr int VEC = Elem<T>::kVec;
     constexpr int NPV = V::kPairs;    // float2 pairs per 16-byte vector
     constexpr int NP = kWJ * NPV;     // pairs per thread and chunk
     extern __shared__ __align__(128) unsigned char smem[];
-    WShared &sh = *reinterpret_cast<WShared *>(smem + (size_t)kQStages * kChunkBytes);
+    WShared &sh = *reinterpret_cast<WShared *>(smem + (size_t)kGroups * kRingBytes);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gid = tid / kGThreads, tg = tid % kGThreads;  // group, and thread within it
+    unsigned char *ring = smem + (size_t)gid * kRingBytes;
+    unsigned long long *full = sh.full[gid];
     const ciar_quantify_out &o = a.out;
 
     if (tid == 0) {
 #pragma unroll
-        for (int s = 0; s < kQStages; ++s) mbar_init(&sh.full[s], 1);
+        for (int s = 0; s < kGroups * kQStages; ++s) mbar_init(&sh.full[0][0] + s, 1);
         sh.abort = 0;
         mbar_init_fence();
     }
     __syncthreads();
 
     const int nvec = a.n / VEC;
-    const int nch = (nvec + kChunkVecs - 1) / kChunkVecs;
+    const int nch_row = (nvec + kChunkVecs - 1) / kChunkVecs;
+    const int nch = (nch_row - gid + kGroups - 1) / kGroups;  // this group's chunks of a row: gid, gid + 2, ...
     const int nk = (int)((a.rows - blockIdx.x + gridDim.x - 1) / gridDim.x);  // rows this CTA walks (the grid never exceeds the rows)
     auto row_of = [&](int k) -> int64_t { return blockIdx.x + (int64_t)k * gridDim.x; };
     // the next row at or after `from` that has something to quantify (-1: none left)
@@ -94,17 +107,19 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
         it.pass = 0;
         it.k = next_active(it.k + 1);
     };
-    // thread 0: asks for the chunk of item `it`, the g-th of this CTA's walk, into stage g mod 3
+    // a group's first thread: asks for the chunk of item `it`, the g-th of the group's walk, into stage g mod 3
     auto issue = [&](const Item &it, int g) {
         if (it.k < 0) return;
         int64_t pr;
         map_row(a.rm, row_of(it.k), pr);
-        const int v0 = it.c * kChunkVecs;
+        const int v0 = (it.c * kGroups + gid) * kChunkVecs;
         const uint32_t bytes = (uint32_t)min(kChunkVecs, nvec - v0) * 16u;
         const int s = g % kQStages;
-        mbar_arrive_expect_tx(&sh.full[s], bytes);
-        bulk_copy_g2s(smem + (size_t)s * kChunkBytes,
-                      reinterpret_cast<const T *>(a.logits) + a.vb + pr * a.row_stride + (int64_t)v0 * VEC, bytes, &sh.full[s]);
+        mbar_arrive_expect_tx(&full[s], bytes);
+        // pass A's lines are wanted once more, by pass B, which is their last use
+        bulk_copy_g2s_hint(ring + (size_t)s * kChunkBytes,
+                           reinterpret_cast<const T *>(a.logits) + a.vb + pr * a.row_stride + (int64_t)v0 * VEC, bytes, &full[s],
+                           it.pass == 0 ? l2_policy_evict_last() : l2_policy_evict_first());
     };
     // Every warp finishes one parked row.  Only the row parked last can have a list longer than its slot
     // (such a row is finished at once); the slot's part then moves next to the rest in the shared buffer.
@@ -127,36 +142,41 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
     if (tid == 0) retire_skipped(0, k);
 #pragma unroll 1
     for (int i = 0; i < kQStages; ++i) {
-        if (tid == 0) issue(pit, i);
+        if (tg == 0) issue(pit, i);
         advance(pit);
     }
 
     int g = 0, filled = 0, rp = 0;  // items swept, rows parked, parity of the rows swept
     bool aborted = false;
 
-    // One pass over the chunks of the row being swept: waits for each chunk, lets `body` sweep it, and after
-    // a barrier (every thread has read the stage) asks for the chunk three further on.  False: a copy never came.
-    auto for_chunks = [&](auto &&body) -> bool {
+    // One pass of this group over its chunks of the row being swept: waits for each chunk, lets `body` sweep it,
+    // and after the group's barrier (all its threads have read the stage) asks for the chunk three further on.
+    // `body` gets a compile-time flag saying that the chunk is a whole one: every thread then owns kWJ vectors of
+    // it.  Once a copy has failed to arrive nothing is waited for any more; the CTA leaves at its next barrier.
+    auto for_chunks = [&](auto &&body) {
 #pragma unroll 1
-        for (int c = 0; c < nch; ++c) {
+        for (int cl = 0; cl < nch; ++cl) {
             const int s = g % kQStages;
-            const unsigned char *stage = smem + (size_t)s * kChunkBytes;
+            const unsigned char *stage = ring + (size_t)s * kChunkBytes;
+            const int c = cl * kGroups + gid;
             const int v0 = c * kChunkVecs;
-            int nj = (min(kChunkVecs, nvec - v0) - tid + kQThreads - 1) / kQThreads;
-            nj = nj < 0 ? 0 : (nj > kWJ ? kWJ : nj);
-            if (!mbar_wait_bounded(&sh.full[s], (uint32_t)(g / kQStages) & 1u, kWaitCycles)) sh.abort = 1;
-            body(c, stage, v0, nj, c == nch - 1);
+            if (!sh.abort && !mbar_wait_bounded(&full[s], (uint32_t)(g / kQStages) & 1u, kWaitCycles)) sh.abort = 1;
+            if (nvec - v0 >= kChunkVecs) {
+                body(std::true_type(), c, stage, v0, kWJ);
+            } else {
+                int nj = (nvec - v0 - tg + kGThreads - 1) / kGThreads;
+                nj = nj < 0 ? 0 : nj;
+                body(std::false_type(), c, stage, v0, nj);
+            }
             __syncwarp();
-            named_bar_sync(kBarRow, kQThreads);
-            if (sh.abort) return false;
-            if (tid == 0) {
+            named_bar_sync(kBarRow + gid, kGThreads);
+            if (tg == 0 && !sh.abort) {
                 fence_proxy_async_smem();
                 issue(pit, g + kQStages);
             }
             advance(pit);
             ++g;
         }
-        return true;
     };
 
     while (k >= 0) {
@@ -171,11 +191,12 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
             float m_w = -INFINITY;
             double zd = 0.0, td = 0.0;
             int cnt = 0, wchunk = 0;  // codes equal to the maximum (counted, not summed); first chunk holding it
-            const bool ok = for_chunks([&](int c, const unsigned char *stage, int, int nj, bool last) {
+            for_chunks([&](auto whole, int c, const unsigned char *stage, int, int nj) {
+                constexpr bool W = decltype(whole)::value;
                 typename V::Max mx = V::max_init();
 #pragma unroll
                 for (int j = 0; j < kWJ; ++j)
-                    if (j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * kQThreads));
+                    if (W || j < nj) mx = V::fold_max(mx, stage_vec(stage, tg + j * kGThreads));
                 const float wmc = warp_redux_max(V::max_value(mx));
                 if (wmc > m_w) {  // the maximum moves: what was summed so far is rescaled to it (in double)
                     if (m_w > -INFINITY) {
@@ -197,9 +218,9 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                         const float2 L2 = f2(kLog2e), nm2 = f2(-m2w);
 #pragma unroll
                         for (int j = 0; j < kWJ; ++j) {
-                            if (j < nj) {
+                            if (W || j < nj) {
                                 float2 cc[NPV];
-                                V::pairs(stage_vec(stage, tid + j * kQThreads), cc);
+                                V::pairs(stage_vec(stage, tg + j * kGThreads), cc);
 #pragma unroll
                                 for (int q = 0; q < NPV; ++q) {
                                     const float2 d = __ffma2_rn(cc[q], L2, nm2);
@@ -214,7 +235,7 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                     if (!(ts == ts)) {  // a -inf logit or a real NaN: the product of such a code is taken as 0 (a NaN still shows in zs)
                         ts = 0.f;
                         for (int j = 0; j < nj; ++j) {
-                            const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+                            const T *v = reinterpret_cast<const T *>(stage + (size_t)(tg + j * kGThreads) * 16);
 #pragma unroll
                             for (int q = 0; q < VEC; ++q) {
                                 const float d = fmaf(Elem<T>::widen(v[q]), kLog2e, -m2w);
@@ -228,7 +249,7 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                         const float e0w = ex2_approx(fmaf(m_w, kLog2e, -m2w));
                         float zz = 0.f;
                         for (int j = 0; j < nj; ++j) {
-                            const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+                            const T *v = reinterpret_cast<const T *>(stage + (size_t)(tg + j * kGThreads) * 16);
 #pragma unroll
                             for (int q = 0; q < VEC; ++q) {
                                 const float ev = ex2_approx(fmaf(Elem<T>::widen(v[q]), kLog2e, -m2w));
@@ -240,31 +261,31 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                     zd += (double)zs;
                     td += (double)ts;
                 }
-                if (last) {  // the warp's share of the row's statistics
-                    const double zw = warp_sum_d(zd), tw = warp_sum_d(td);
-                    int cw = cnt;
-#pragma unroll
-                    for (int ofs = 16; ofs > 0; ofs >>= 1) cw += __shfl_xor_sync(0xffffffffu, cw, ofs);
-                    if (lane == 0) {
-                        sh.wm[warp] = m_w;
-                        sh.wz[warp] = zw;
-                        sh.wt[warp] = tw;
-                        sh.wcnt[warp] = cw;
-                        sh.wchunk[warp] = wchunk;
-                    }
-                }
             });
-            if (!ok) {
-                aborted = true;
-                break;
+            // the warp's share of the row's statistics
+            const double zw = warp_sum_d(zd), tw = warp_sum_d(td);
+            int cw = cnt;
+#pragma unroll
+            for (int ofs = 16; ofs > 0; ofs >>= 1) cw += __shfl_xor_sync(0xffffffffu, cw, ofs);
+            if (lane == 0) {
+                sh.wm[warp] = m_w;
+                sh.wz[warp] = zw;
+                sh.wt[warp] = tw;
+                sh.wcnt[warp] = cw;
+                sh.wchunk[warp] = wchunk;
             }
+        }
+        __syncthreads();  // both groups are through pass A: the warps' shares are out
+        if (sh.abort) {
+            aborted = true;
+            break;
         }
         // ---- the row's statistics from the warps' (lane w joins warp w's share, rescaled to the row maximum)
         float m, m2, zf, c0, th, th_log, r;
         int status = 0;
         bool classify, series, direct;
         {
-            const int w = lane & (kQWarps - 1);
+            const int w = lane & (kWWarps - 1);
             const float mw = sh.wm[w];
             m = warp_redux_max(mw);
             m2 = m * kLog2e;
@@ -288,7 +309,7 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                 }
             }
 #pragma unroll
-            for (int ofs = kQWarps / 2; ofs > 0; ofs >>= 1) {
+            for (int ofs = kWWarps / 2; ofs > 0; ofs >>= 1) {
                 zc += __shfl_xor_sync(0xffffffffu, zc, ofs);
                 tc += __shfl_xor_sync(0xffffffffu, tc, ofs);
                 nc += __shfl_xor_sync(0xffffffffu, nc, ofs);
@@ -330,13 +351,12 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
             }
         }
         // ---- pass B: with the maximum and the sum of exponentials known
-        bool ok;
         if (classify) {
             // an unusable row: what it contains, exactly as the row-status bits are defined
             int has_nan = 0, has_finite = 0;
-            ok = for_chunks([&](int, const unsigned char *stage, int, int nj, bool last) {
+            for_chunks([&](auto, int, const unsigned char *stage, int, int nj) {
                 for (int j = 0; j < nj; ++j) {
-                    const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+                    const T *v = reinterpret_cast<const T *>(stage + (size_t)(tg + j * kGThreads) * 16);
 #pragma unroll
                     for (int q = 0; q < VEC; ++q) {
                         const float c = Elem<T>::widen(v[q]);
@@ -344,17 +364,11 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                         if (c == c && fabsf(c) != INFINITY) has_finite = 1;
                     }
                 }
-                if (last) {
-                    if (has_nan) sh.bad_nan[rp] = 1;
-                    if (has_finite) sh.bad_finite[rp] = 1;
-                }
             });
-            status = 0;
-            if (sh.bad_nan[rp]) status |= CIAR_ROW_NAN;
-            if (!sh.bad_finite[rp]) status |= CIAR_ROW_NO_FINITE;
-            if (!status) status = CIAR_ROW_NAN;  // sums overflowed without any single bad logit
+            if (has_nan) sh.bad_nan[rp] = 1;
+            if (has_finite) sh.bad_finite[rp] = 1;
         } else if (status) {
-            ok = for_chunks([&](int, const unsigned char *, int, int, bool) {});  // the chunks were asked for already
+            for_chunks([&](auto, int, const unsigned char *, int, int) {});  // the chunks were asked for already
         } else {
             // the first chunk in which this warp met the row maximum holds its candidates for the arg-max
             const int amchunk = sh.wm[warp] == m ? sh.wchunk[warp] : -1;
@@ -362,16 +376,17 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                 if (c != amchunk) return;
                 int best = INT_MAX;
                 for (int j = nj - 1; j >= 0; --j) {
-                    const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+                    const T *v = reinterpret_cast<const T *>(stage + (size_t)(tg + j * kGThreads) * 16);
 #pragma unroll
                     for (int q = VEC - 1; q >= 0; --q)
-                        if (Elem<T>::widen(v[q]) == m) best = (v0 + tid + j * kQThreads) * VEC + q;
+                        if (Elem<T>::widen(v[q]) == m) best = (v0 + tg + j * kGThreads) * VEC + q;
                 }
                 if (best != INT_MAX) atomicMin(&sh.argmin[rp], best);
             };
             if (series) {
                 double a2 = 0.0, a3 = 0.0, a4 = 0.0;  // power sums of (e - c0) over the row
-                ok = for_chunks([&](int c, const unsigned char *stage, int v0, int nj, bool last) {
+                for_chunks([&](auto whole, int c, const unsigned char *stage, int v0, int nj) {
+                    constexpr bool W = decltype(whole)::value;
                     arg_max(c, stage, v0, nj);
                     typename V::Max mx = V::max_init();
                     float2 e[NP];
@@ -379,8 +394,8 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                         const float2 L2 = f2(kLog2e), nm2 = f2(-m2);
 #pragma unroll
                         for (int j = 0; j < kWJ; ++j) {
-                            if (j < nj) {
-                                const uint4 &vv = stage_vec(stage, tid + j * kQThreads);
+                            if (W || j < nj) {
+                                const uint4 &vv = stage_vec(stage, tg + j * kGThreads);
                                 mx = V::fold_max(mx, vv);
                                 float2 cc[NPV];
                                 V::pairs(vv, cc);
@@ -423,7 +438,7 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                     const float2 nc0 = f2(-c0);
 #pragma unroll
                     for (int i = 0; i < NP; ++i) {
-                        if (i / NPV < nj) {
+                        if (W || i / NPV < nj) {
                             const float2 y = __fadd2_rn(e[i], nc0);
                             const float2 y2 = __fmul2_rn(y, y);
                             T2 = __fadd2_rn(T2, y2);
@@ -434,26 +449,24 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                     a2 += (double)(T2.x + T2.y);
                     a3 += (double)(T3.x + T3.y);
                     a4 += (double)(T4.x + T4.y);
-                    if (last) {
-                        const double s2 = warp_sum_d(a2), s3 = warp_sum_d(a3), s4 = warp_sum_d(a4);
-                        if (lane == 0) {
-                            sh.ws[warp][0] = s2;
-                            sh.ws[warp][1] = s3;
-                            sh.ws[warp][2] = s4;
-                        }
-                    }
                 });
+                const double s2 = warp_sum_d(a2), s3 = warp_sum_d(a3), s4 = warp_sum_d(a4);
+                if (lane == 0) {
+                    sh.ws[warp][0] = s2;
+                    sh.ws[warp][1] = s3;
+                    sh.ws[warp][2] = s4;
+                }
             } else {
                 // both bounds of every code
                 const DirectConst dc = make_direct_const(r, a.n);
                 const float invz = 1.0f / zf;
                 double acc[5] = { 0.0, 0.0, 0.0, 0.0, 0.0 };
-                ok = for_chunks([&](int c, const unsigned char *stage, int v0, int nj, bool last) {
+                for_chunks([&](auto, int c, const unsigned char *stage, int v0, int nj) {
                     arg_max(c, stage, v0, nj);
                     float ps[5] = { 0.f, 0.f, 0.f, 0.f, 0.f };
 #pragma unroll 1
                     for (int j = 0; j < nj; ++j) {
-                        const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+                        const T *v = reinterpret_cast<const T *>(stage + (size_t)(tg + j * kGThreads) * 16);
                         float cc[VEC];
                         Elem<T>::load(v, cc);
 #pragma unroll
@@ -473,19 +486,24 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
                     }
 #pragma unroll
                     for (int q = 0; q < 5; ++q) acc[q] += (double)ps[q];
-                    if (last) {
-#pragma unroll
-                        for (int q = 0; q < 5; ++q) {
-                            const double tot = warp_sum_d(acc[q]);
-                            if (lane == 0) sh.ws[warp][q] = tot;
-                        }
-                    }
                 });
+#pragma unroll
+                for (int q = 0; q < 5; ++q) {
+                    const double tot = warp_sum_d(acc[q]);
+                    if (lane == 0) sh.ws[warp][q] = tot;
+                }
             }
         }
-        if (!ok) {
+        __syncthreads();  // both groups are through pass B: the warps' sums, the list and the arg-max are complete
+        if (sh.abort) {
             aborted = true;
             break;
+        }
+        if (classify) {
+            status = 0;
+            if (sh.bad_nan[rp]) status |= CIAR_ROW_NAN;
+            if (!sh.bad_finite[rp]) status |= CIAR_ROW_NO_FINITE;
+            if (!status) status = CIAR_ROW_NAN;  // sums overflowed without any single bad logit
         }
         // ---- park the rest: the route's sums (series: powers 2, 3, 4; direct: pl, dd, pl^2, pl dd, dd^2)
         if (tid < kQWarps * 8 && (tid & 3) != 0) {
@@ -493,7 +511,7 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
             const int q = slot == 1 ? 0 : slot == 5 ? 1 : slot == 2 ? 2 : slot == 6 ? 3 : slot == 3 ? 4 : -1;
             double tot = 0.0;
             if (!status && q >= 0 && (q < 3 || direct))
-                for (int ww = 0; ww < kQWarps; ++ww) tot += sh.ws[ww][q];
+                for (int ww = 0; ww < kWWarps; ++ww) tot += sh.ws[ww][q];
             const float hi = (float)tot;
             pk.wsum[wrow][slot] = wrow == 0 ? hi : (wrow == 1 ? (float)(tot - (double)hi) : 0.f);
         }
@@ -514,18 +532,19 @@ __global__ void __launch_bounds__(kQThreads, 2) quantify_wide_kernel(const __gri
     }
     if (filled > 0) finish_parked(filled);
 
-    if (aborted && tid == 0) {
+    if (aborted && tg == 0) {
         // A copy never arrived.  Mark this row and the rest of this CTA's rows, then give the copies
         // still in flight a last bounded chance to land before the CTA leaves.
-        for (int k2 = k; k2 < nk; ++k2) write_unusable(o, row_of(k2), CIAR_ROW_TIMEOUT);
+        if (tid == 0)
+            for (int k2 = k; k2 < nk; ++k2) write_unusable(o, row_of(k2), CIAR_ROW_TIMEOUT);
         for (int i = 0; i < kQStages; ++i)
-            mbar_wait_bounded(&sh.full[(g + i) % kQStages], (uint32_t)((g + i) / kQStages) & 1u, kDrainCycles);
+            mbar_wait_bounded(&full[(g + i) % kQStages], (uint32_t)((g + i) / kQStages) & 1u, kDrainCycles);
     }
 }
 
 cudaError_t launch_wide(const QuantifyArgs &a, int dtype, cudaStream_t stream)
 {
-    constexpr size_t smem = (size_t)kQStages * kChunkBytes + sizeof(WShared);
+    constexpr size_t smem = (size_t)kGroups * kRingBytes + sizeof(WShared);
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
@@ -538,10 +557,10 @@ cudaError_t launch_wide(const QuantifyArgs &a, int dtype, cudaStream_t stream)
         if (err != cudaSuccess) return err;
         configured[dev] = true;
     }
-    const int64_t cap = (int64_t)sm_count() * 2;
+    const int64_t cap = (int64_t)sm_count();
     const unsigned grid = (unsigned)(a.rows < cap ? a.rows : cap);
-    if (dtype == CIAR_F32) quantify_wide_kernel<float><<<grid, kQThreads, smem, stream>>>(a);
-    else quantify_wide_kernel<__nv_bfloat16><<<grid, kQThreads, smem, stream>>>(a);
+    if (dtype == CIAR_F32) quantify_wide_kernel<float><<<grid, kWThreads, smem, stream>>>(a);
+    else quantify_wide_kernel<__nv_bfloat16><<<grid, kWThreads, smem, stream>>>(a);
     count_launch();
     return cudaGetLastError();
 }

@@ -63,6 +63,31 @@ __device__ __forceinline__ void bulk_copy_g2s(void *dst_smem, const void *src_gm
                  : "memory");
 }
 
+// L2 eviction policies for a bulk copy: keep the lines (they are read once more soon) / drop them first.
+__device__ __forceinline__ unsigned long long l2_policy_evict_last()
+{
+    unsigned long long p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+__device__ __forceinline__ unsigned long long l2_policy_evict_first()
+{
+    unsigned long long p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+// bulk_copy_g2s with an L2 eviction policy for the lines it reads
+__device__ __forceinline__ void bulk_copy_g2s_hint(void *dst_smem, const void *src_gmem, uint32_t bytes, unsigned long long *bar,
+                                                   unsigned long long policy)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+                     smem_addr(dst_smem)),
+                 "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar)), "l"(policy)
+                 : "memory");
+}
+
 // Orders earlier generic-proxy accesses of shared memory before later asynchronous-proxy ones.
 __device__ __forceinline__ void fence_proxy_async_smem()
 {
