@@ -16,6 +16,7 @@
 // drop them.
 #include <type_traits>
 
+#include "online_stats.cuh"
 #include "quantify_finish.cuh"
 
 namespace ciar {
@@ -188,91 +189,22 @@ __global__ void __launch_bounds__(kWThreads, 1) quantify_wide_kernel(const __gri
         }
         // ---- pass A: every warp's running maximum, and per lane the sums of exp and exp * exponent relative to it
         {
-            float m_w = -INFINITY;
-            double zd = 0.0, td = 0.0;
-            int cnt = 0, wchunk = 0;  // codes equal to the maximum (counted, not summed); first chunk holding it
+            OnlineStats st;
+            st.reset();
             for_chunks([&](auto whole, int c, const unsigned char *stage, int, int nj) {
-                constexpr bool W = decltype(whole)::value;
-                typename V::Max mx = V::max_init();
-#pragma unroll
-                for (int j = 0; j < kWJ; ++j)
-                    if (W || j < nj) mx = V::fold_max(mx, stage_vec(stage, tg + j * kGThreads));
-                const float wmc = warp_redux_max(V::max_value(mx));
-                if (wmc > m_w) {  // the maximum moves: what was summed so far is rescaled to it (in double)
-                    if (m_w > -INFINITY) {
-                        const float m2o = m_w * kLog2e;
-                        const double dl = (double)m2o - (double)(wmc * kLog2e);  // change of every exponent
-                        const double f = exp2(dl);
-                        const double tot = zd + (double)cnt * (double)ex2_approx(fmaf(m_w, kLog2e, -m2o));
-                        td = f * (td + dl * tot);
-                        zd = tot * f;
-                        cnt = 0;
-                    }
-                    m_w = wmc;
-                    wchunk = c;
-                }
-                if (m_w > -INFINITY) {
-                    const float m2w = m_w * kLog2e;
-                    float2 z2 = f2(0.f), t2 = f2(0.f);
-                    {
-                        const float2 L2 = f2(kLog2e), nm2 = f2(-m2w);
-#pragma unroll
-                        for (int j = 0; j < kWJ; ++j) {
-                            if (W || j < nj) {
-                                float2 cc[NPV];
-                                V::pairs(stage_vec(stage, tg + j * kGThreads), cc);
-#pragma unroll
-                                for (int q = 0; q < NPV; ++q) {
-                                    const float2 d = __ffma2_rn(cc[q], L2, nm2);
-                                    const float2 ev = make_float2(ex2_approx(d.x), ex2_approx(d.y));  // a NaN logit poisons the sums on purpose
-                                    z2 = __fadd2_rn(z2, ev);
-                                    t2 = __ffma2_rn(ev, d, t2);  // 0 * -inf = NaN for a -inf logit: redone below
-                                }
-                            }
-                        }
-                    }
-                    float zs = z2.x + z2.y, ts = t2.x + t2.y;
-                    if (!(ts == ts)) {  // a -inf logit or a real NaN: the product of such a code is taken as 0 (a NaN still shows in zs)
-                        ts = 0.f;
-                        for (int j = 0; j < nj; ++j) {
-                            const T *v = reinterpret_cast<const T *>(stage + (size_t)(tg + j * kGThreads) * 16);
-#pragma unroll
-                            for (int q = 0; q < VEC; ++q) {
-                                const float d = fmaf(Elem<T>::widen(v[q]), kLog2e, -m2w);
-                                ts = fmaf(ex2_approx(d), fmaxf(d, kNegHuge), ts);
-                            }
-                        }
-                    }
-                    if (wmc == m_w) {
-                        // This chunk holds codes equal to the warp's maximum.  A term near 1 would cost the small terms
-                        // their low bits, so the sums are formed again without such terms; they are counted instead.
-                        const float e0w = ex2_approx(fmaf(m_w, kLog2e, -m2w));
-                        float zz = 0.f;
-                        for (int j = 0; j < nj; ++j) {
-                            const T *v = reinterpret_cast<const T *>(stage + (size_t)(tg + j * kGThreads) * 16);
-#pragma unroll
-                            for (int q = 0; q < VEC; ++q) {
-                                const float ev = ex2_approx(fmaf(Elem<T>::widen(v[q]), kLog2e, -m2w));
-                                if (ev == e0w) ++cnt; else zz += ev;
-                            }
-                        }
-                        zs = zz;
-                    }
-                    zd += (double)zs;
-                    td += (double)ts;
-                }
+                online_sweep<T, kGThreads, kWJ, decltype(whole)::value, true>(st, stage, tg, nj, c);
             });
             // the warp's share of the row's statistics
-            const double zw = warp_sum_d(zd), tw = warp_sum_d(td);
-            int cw = cnt;
+            const double zw = warp_sum_d(st.zd), tw = warp_sum_d(st.td);
+            int cw = st.cnt;
 #pragma unroll
             for (int ofs = 16; ofs > 0; ofs >>= 1) cw += __shfl_xor_sync(0xffffffffu, cw, ofs);
             if (lane == 0) {
-                sh.wm[warp] = m_w;
+                sh.wm[warp] = st.m_w;
                 sh.wz[warp] = zw;
                 sh.wt[warp] = tw;
                 sh.wcnt[warp] = cw;
-                sh.wchunk[warp] = wchunk;
+                sh.wchunk[warp] = st.chunk;
             }
         }
         __syncthreads();  // both groups are through pass A: the warps' shares are out

@@ -9,6 +9,7 @@
 #include <climits>
 
 #include "ciar_internal.h"
+#include "online_stats.cuh"
 #include "stream_common.cuh"
 #include "verify_resample.cuh"
 
@@ -337,6 +338,151 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
     }
 }
 
+// ---- accept, rows wider than the on-chip sweep takes: one pass over a row, 32 KB at a time ("chunks") through
+// the same ring, the statistics kept on line by every warp and joined once per row.
+constexpr int kVWJ = 4;
+constexpr int kVChunkVecs = kVThreads * kVWJ;
+constexpr int kVChunkBytes = kVChunkVecs * 16;
+
+struct VWShared {
+    unsigned long long full[kVStages];
+    float wm[kVWarps];  // per warp: running maximum, sum relative to it, number of codes equal to it
+    double wz[kVWarps];
+    int wcnt[kVWarps];
+    int abort;
+    VParked park[kVPark];
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kVThreads, 2) verify_accept_wide_kernel(const __grid_constant__ VerifyArgs a)
+{
+    constexpr int VEC = Elem<T>::kVec;
+    extern __shared__ __align__(128) unsigned char smem[];
+    VWShared &sh = *reinterpret_cast<VWShared *>(smem + (size_t)kVStages * kVChunkBytes);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+#pragma unroll
+        for (int s = 0; s < kVStages; ++s) mbar_init(&sh.full[s], 1);
+        sh.abort = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+    const int nvec = a.n / VEC;
+    const int nch = (nvec + kVChunkVecs - 1) / kVChunkVecs;
+    const T *tbase = reinterpret_cast<const T *>(a.target) + a.vb;
+    const int total = a.ws.tested[a.rows];  // written by the plan kernel
+    const int stride = gridDim.x;
+    const int mine = blockIdx.x < total ? (total - 1 - (int)blockIdx.x) / stride + 1 : 0;  // rows this CTA walks
+
+    // thread 0: asks for chunk c of this CTA's kr-th row, the g-th chunk of its walk, into stage g mod 3
+    auto issue = [&](int kr, int c, int g) {
+        if (kr >= mine) return;
+        int64_t pr;
+        map_row(a.rm, a.ws.tested[blockIdx.x + kr * stride], pr);
+        const int v0 = c * kVChunkVecs;
+        const uint32_t bytes = (uint32_t)min(kVChunkVecs, nvec - v0) * 16u;
+        const int s = g % kVStages;
+        mbar_arrive_expect_tx(&sh.full[s], bytes);
+        bulk_copy_g2s(smem + (size_t)s * kVChunkBytes, tbase + pr * a.row_stride + (int64_t)v0 * VEC, bytes, &sh.full[s]);
+    };
+    auto finish_parked = [&](int count) {
+        __syncthreads();
+        if (warp < count) accept_row<T>(a, sh.park[warp], lane);
+        __syncthreads();
+    };
+    int pr_k = 0, pr_c = 0;  // the chunk to ask for next, three ahead of the sweep
+    auto advance = [&]() {
+        if (++pr_c == nch) {
+            pr_c = 0;
+            ++pr_k;
+        }
+    };
+#pragma unroll 1
+    for (int i = 0; i < kVStages; ++i) {
+        if (tid == 0) issue(pr_k, pr_c, i);
+        advance();
+    }
+    int k = 0, g = 0, filled = 0;
+    bool aborted = false;
+    for (; k < mine; ++k) {
+        OnlineStats st;
+        st.reset();
+#pragma unroll 1
+        for (int c = 0; c < nch; ++c) {
+            const int s = g % kVStages;
+            const unsigned char *stage = smem + (size_t)s * kVChunkBytes;
+            const int v0 = c * kVChunkVecs;
+            // once a copy has failed to arrive nothing is waited for any more; the CTA leaves after this row's barrier
+            if (!sh.abort && !mbar_wait_bounded(&sh.full[s], (uint32_t)(g / kVStages) & 1u, kWaitCycles)) sh.abort = 1;
+            if (nvec - v0 >= kVChunkVecs) {
+                online_sweep<T, kVThreads, kVWJ, true, false>(st, stage, tid, kVWJ, c);
+            } else {
+                int nj = (nvec - v0 - tid + kVThreads - 1) / kVThreads;
+                nj = nj < 0 ? 0 : nj;
+                online_sweep<T, kVThreads, kVWJ, false, false>(st, stage, tid, nj, c);
+            }
+            __syncwarp();
+            __syncthreads();  // every thread has read the stage
+            if (tid == 0 && !sh.abort) {
+                fence_proxy_async_smem();
+                issue(pr_k, pr_c, g + kVStages);
+            }
+            advance();
+            ++g;
+        }
+        {
+            double zw, tw;
+            int cw;
+            online_warp_totals(st, zw, tw, cw);
+            if (lane == 0) {
+                sh.wm[warp] = st.m_w;
+                sh.wz[warp] = zw;
+                sh.wcnt[warp] = cw;
+            }
+        }
+        __syncthreads();  // the warps' shares are out
+        if (sh.abort) {
+            aborted = true;
+            break;
+        }
+        if (warp == 0) {
+            // Park the row in the form the finishing routine reads: the sum as a float pair (high part in warp
+            // 0's place, the remainder in warp 1's, zeros in the others), so that its double sum is the sum.
+            float m;
+            double zc, tc;
+            int nc;
+            online_join<kVWarps>(sh.wm, sh.wz, nullptr, sh.wcnt, lane, m, zc, tc, nc);
+            VParked &pk = sh.park[filled];
+            const float hi = (float)zc;
+            if (lane < kVWarps) pk.wz[lane] = lane == 0 ? hi : (lane == 1 ? (float)(zc - (double)hi) : 0.f);
+            if (lane == 0) {
+                pk.lr = a.ws.tested[blockIdx.x + k * stride];
+                pk.m = m;
+                pk.e0 = ex2_approx(fmaf(m, kLog2e, -(m * kLog2e)));
+                pk.nmax = nc;
+            }
+        }
+        if (++filled == kVPark) {
+            finish_parked(filled);
+            filled = 0;
+        }
+    }
+    if (filled > 0) finish_parked(filled);
+    if (aborted && tid == 0) {
+        // A copy never arrived: the rows this CTA still owed are marked, and the copies in flight
+        // get a last bounded chance to land before the CTA leaves.
+        uint8_t *accept_arr = a.out.accept ? a.out.accept : a.ws.accept;
+        for (int k2 = k; k2 < mine; ++k2) {
+            const int64_t lr = a.ws.tested[blockIdx.x + k2 * stride];
+            accept_arr[lr] = 0;
+            a.ws.tq_sum[lr] = __int_as_float(0x7fc00000);
+            if (a.out.row_status) a.out.row_status[lr] = CIAR_ROW_TIMEOUT;
+        }
+        for (int i = 0; i < kVStages; ++i)
+            mbar_wait_bounded(&sh.full[(g + i) % kVStages], (uint32_t)((g + i) / kVStages) & 1u, kDrainCycles);
+    }
+}
+
 // ---- window: accepted length and, for a rejected window, the residual sample of its first rejected row
 template <typename T>
 __global__ void __launch_bounds__(kWinThreads) verify_window_kernel(VerifyArgs a)
@@ -424,6 +570,27 @@ cudaError_t launch_accept(const VerifyArgs &a, cudaStream_t stream, bool full)
 }
 
 template <typename T>
+cudaError_t launch_accept_wide(const VerifyArgs &a, cudaStream_t stream)
+{
+    constexpr size_t smem = (size_t)kVStages * kVChunkBytes + sizeof(VWShared);
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
+        err = cudaFuncSetAttribute(verify_accept_wide_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        configured[dev] = true;
+    }
+    const int64_t cap = (int64_t)sm_count() * 2;
+    const unsigned grid = (unsigned)(a.rows < cap ? a.rows : cap);
+    verify_accept_wide_kernel<T><<<grid, kVThreads, smem, stream>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <typename T>
 cudaError_t launch_all(const VerifyArgs &a, cudaStream_t stream)
 {
     cudaError_t err = cudaMemsetAsync(a.ws.tested + a.rows, 0, sizeof(int32_t), stream);
@@ -436,7 +603,8 @@ cudaError_t launch_all(const VerifyArgs &a, cudaStream_t stream)
     const int nvec = a.n / Elem<T>::kVec;
     const int jv = nvec <= kVThreads ? 1 : (nvec <= 2 * kVThreads ? 2 : (nvec <= 4 * kVThreads ? 4 : 8));
     const bool full = nvec == kVThreads * jv;
-    switch (jv) {
+    if (a.n > 16384) err = launch_accept_wide<T>(a, stream);
+    else switch (jv) {
     case 1: err = launch_accept<T, 1>(a, stream, full); break;
     case 2: err = launch_accept<T, 2>(a, stream, full); break;
     case 4: err = launch_accept<T, 4>(a, stream, full); break;
@@ -459,7 +627,7 @@ bool verify_stream_eligible(const VerifyArgs &a, int dtype)
     if (!a.draft_row_max || !a.draft_sum_exp) return false;
     if (a.vb % vec != 0 || a.n % vec != 0) return false;
     if (a.rows >= INT_MAX) return false;
-    return a.n >= 2048 && a.n <= 16384;
+    return a.n >= 2048 && a.n <= (1 << 28);
 }
 
 cudaError_t launch_verify_stream(const VerifyArgs &a, int dtype, cudaStream_t stream)

@@ -266,6 +266,32 @@ def test_verify_with_quantify_stats_and_slice(ciar, dtype):
     assert ref.accept[5] == 0 and ref.p_draft_tok[5] == 0.0
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("vocab,vb,n", [(40000, 0, 40000), (70000, 1024, 50008)])
+def test_verify_wide_rows(ciar, vocab, vb, n, dtype):
+    """The streaming verifier on rows wider than its on-chip sweep takes (one pass, chunk by chunk, last chunk
+    ragged), draft statistics from the quantifier; degenerate target rows among ordinary ones."""
+    rows, window = 48, 8
+    draft, target, tok, flag, ua, ur = _verify_case(rows, vocab, dtype, window, seed=vocab + 3, sigma=0.7)
+    tok = np.clip(tok, vb, vb + n - 1).astype(np.int32)
+    flag[0] = 1
+    target[3] = draft[3]  # identical rows: always accepted
+    target[9] = float("-inf")  # target without a finite code
+    target[17, vb + n - 1] = float("nan")
+    target[20, vb: vb + n - 4000] = float("-inf")  # the first chunks hold nothing finite
+    target[26, vb + 5] = 60.0  # maximum in the first chunk
+    target[27, vb + n - 2] = 60.0  # maximum in the last one
+    target[30, [vb + 7, vb + 20000, vb + n - 1]] = 40.0  # equal maxima in three chunks
+    dd, td = draft.cuda(), target.cuda()
+    qo = ciar.QuantifyOut.allocate(rows, "cuda")
+    ciar.quantify(dd, ciar.IntervalParams(r_scalar=0.2, tau=1e-4), qo, vb, n)
+    for mode in (oracle.VERIFY_ANCHORED, oracle.VERIFY_ALL):
+        ref, out, rep = pu.check_verify(draft, target, tok, flag, ua, ur, window, mode, vb, n,
+                                        draft_stats=(qo.row_max, qo.sum_exp), draft_dev=dd, target_dev=td)
+    st = out.row_status.cpu().numpy()  # of the run that tests every row
+    assert st[9] & oracle.ROW_NO_FINITE and st[17] & oracle.ROW_NAN
+
+
 def test_verify_degenerate_rows(ciar):
     v, window = 264, 4
     draft, target, tok, flag, ua, ur = _verify_case(16, v, torch.float32, window, seed=4)
