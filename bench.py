@@ -195,6 +195,8 @@ def run_ours(args):
     barrier(world)
     clocks = sampler.stop()
     launches = ciar.launch_count() - launches0
+    if graph is not None:
+        launches = steps * launches_per_step  # replays do not pass through the library's counter
     total_ms = max_over_ranks(t_start.elapsed_time(t_end), world)
     q_ms = float(np.mean([ev[k][0].elapsed_time(ev[k][1]) for k in range(K)]))
     v_ms = float(np.mean([ev[k][1].elapsed_time(ev[k][2]) for k in range(K)]))
@@ -319,6 +321,13 @@ def run_decode(args):
     state = ciar.DecodeState.allocate(req, seq, dev)
     ws = ciar.alloc_workspace(req * wl.window, wl.window, dev)
 
+    def one_step():
+        ciar.decode_step(state, inp.draft, inp.target, inp.tokens, inp.u_accept, inp.u_resample, params, wl.window,
+                         ciar.VERIFY_ANCHORED, ws, wl.valid_begin, wl.n_valid)
+
+    graph = None
+    launches_per_step = None
+
     def loop(record):
         ciar.decode_init(state, 0)
         events = []
@@ -327,8 +336,10 @@ def run_decode(args):
             if record:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-            ciar.decode_step(state, inp.draft, inp.target, inp.tokens, inp.u_accept, inp.u_resample, params, wl.window,
-                             ciar.VERIFY_ANCHORED, ws, wl.valid_begin, wl.n_valid)
+            if graph is not None:
+                graph.replay()  # the step's launches, recorded once (every argument lives on the device)
+            else:
+                one_step()
             if record:
                 e1.record()
                 events.append((e0, e1))
@@ -341,6 +352,21 @@ def run_decode(args):
 
     loop(False)  # warm-up: one whole generation
     torch.cuda.synchronize()
+    if args.decode_graph:
+        # ciar_decode_step allocates nothing and never synchronises, so a caller may record it in a CUDA graph
+        n0 = ciar.launch_count()
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            one_step()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        launches_per_step = ciar.launch_count() - n0
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            one_step()
+        loop(False)  # warm-up of the replays
+        torch.cuda.synchronize()
     sampler = ClockSampler(dev.index or 0)
     launches0 = ciar.launch_count()
     sampler.start()
@@ -352,6 +378,8 @@ def run_decode(args):
     barrier(world)
     clocks = sampler.stop()
     launches = ciar.launch_count() - launches0
+    if graph is not None:
+        launches = steps * launches_per_step  # replays do not pass through the library's counter
     total_ms = max_over_ranks(t0.elapsed_time(t1), world)
     cnt = state.counters.cpu().numpy()
     # steps after the last request finished do no work but are inside the timed region: count only useful ones
@@ -365,6 +393,7 @@ def run_decode(args):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "decode", "requests_per_gpu": req, "seq_len": seq, "vocab": wl.vocab, "logits": wl.dtype,
                    "window": wl.window, "verify_mode": "anchored", "radius": "per_row", "tau": wl.tau,
+                   "launch": "cuda graph replay" if graph is not None else "direct",
                    "l2": "pools of %.1f GB, rows touched once" % (2 * req * seq * wl.vocab * wl.elem_bytes / 1e9)},
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
@@ -426,6 +455,8 @@ def main():
     ap.add_argument("--decode-requests", type=int, default=0, help="decode workload: concurrent requests (default 256)")
     ap.add_argument("--images", type=int, default=0,
                     help="images of the workload (default: the workload's own); a smaller batch for profiler captures")
+    ap.add_argument("--decode-graph", action=argparse.BooleanOptionalAction, default=True,
+                    help="decode workload: replay each step from a CUDA graph (default) or launch it directly")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
