@@ -11,8 +11,8 @@ namespace ciar {
 
 namespace {
 
-constexpr int kQThreads = 512;
-constexpr int kQWarps = kQThreads / 32;
+constexpr int kQThreads = 512;           // most threads a CTA of the streaming quantifiers has
+constexpr int kQWarps = kQThreads / 32;  // (the parked form is laid out for that many warps)
 constexpr int kQStages = 3;
 constexpr int kBarRow = 1;                       // named barrier of the row sweeps
 constexpr long long kWaitCycles = 2000000000ll;  // bound of a wait for a row (about a second)
@@ -120,7 +120,7 @@ __device__ __forceinline__ void write_unusable(const ciar_quantify_out &o, long 
 // Finishes one row whose sums are parked: reduces the per-warp sums, treats the listed codes
 // exactly (one per lane), then does the scalar arithmetic (normalisation step, Omega, Sigma, U,
 // entropy, the flag) and the stores.  Run by one whole warp.
-__device__ __noinline__ void finish_row(const QuantifyArgs &a, const Parked &pk, const float *list, int lane)
+__device__ __noinline__ void finish_row(const QuantifyArgs &a, const Parked &pk, const float *list, int lane, int nw)
 {
     const ciar_quantify_out &o = a.out;
     const long long lr = pk.lr;
@@ -135,7 +135,7 @@ __device__ __noinline__ void finish_row(const QuantifyArgs &a, const Parked &pk,
         constexpr int kSlot[7] = { 0, 4, 1, 5, 2, 6, 3 };
         v[q] = 0.0;
         if (q < 5 || !series) {
-            if (lane < kQWarps) v[q] = (double)pk.wsum[lane][kSlot[q]];
+            if (lane < nw) v[q] = (double)pk.wsum[lane][kSlot[q]];
             v[q] = warp_sum_d(v[q]);
         }
     }

@@ -29,14 +29,15 @@ static_assert(sizeof(QShared) + kQStages * 32768 <= 115712, "two CTAs per SM mus
 
 // FULL: every thread owns exactly JV vectors (the row has 512 * JV of them).  MAPPED: the rows go through a
 // position map (decode mode), so some of them hold nothing to quantify.
-template <typename T, int JV, int MINB, bool FULL, bool MAPPED>
-__global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const __grid_constant__ QuantifyArgs a)
+template <typename T, int NT, int JV, int MINB, bool FULL, bool MAPPED>
+__global__ void __launch_bounds__(NT, MINB) quantify_stream_kernel(const __grid_constant__ QuantifyArgs a)
 {
+    constexpr int NW = NT / 32;  // warps; as many rows are parked before the CTA finishes them, one per warp
     typedef Vec<T> V;
     constexpr int VEC = Elem<T>::kVec;
     constexpr int NPV = V::kPairs;  // float2 pairs per 16-byte vector
     constexpr int NP = JV * NPV;    // pairs per thread
-    constexpr int kStageBytes = kQThreads * JV * 16;
+    constexpr int kStageBytes = NT * JV * 16;
     extern __shared__ __align__(128) unsigned char smem[];
     QShared &sh = *reinterpret_cast<QShared *>(smem + (size_t)kQStages * kStageBytes);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -53,7 +54,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
     const int nvec = a.n / VEC;
     int nj = JV;
     if (!FULL) {
-        nj = (nvec - tid + kQThreads - 1) / kQThreads;
+        nj = (nvec - tid + NT - 1) / NT;
         nj = nj < 0 ? 0 : (nj > JV ? JV : nj);
     }
     const ciar_quantify_out &o = a.out;
@@ -86,7 +87,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
                 __syncwarp();
                 list = big;
             }
-            finish_row(a, p, list, lane);
+            finish_row(a, p, list, lane, NW);
         }
         __syncthreads();
     };
@@ -135,7 +136,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
         typename V::Max mx = V::max_init();
 #pragma unroll
         for (int j = 0; j < JV; ++j)
-            if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * kQThreads));
+            if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * NT));
         const float wm = warp_redux_max(V::max_value(mx));
         if (lane == 0) sh.wmax[turn & 1][warp] = wm;
         if (tid == 0) {
@@ -149,7 +150,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
     if (k >= 0) {
         first_sweep(k, 0);
         __syncwarp();
-        named_bar_sync(kBarRow, kQThreads);
+        named_bar_sync(kBarRow, NT);
         if (sh.abort) aborted = true;
     }
     while (k >= 0 && !aborted) {
@@ -166,7 +167,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             pk.pr = pr;
             pk.rho = a.radius_mode == CIAR_RADIUS_PER_ROW ? reinterpret_cast<const float *>(a.radius)[pr] : a.r_scalar;
         }
-        const float m = warp_redux_max(sh.wmax[par][lane & (kQWarps - 1)]);
+        const float m = warp_redux_max(sh.wmax[par][lane & (NW - 1)]);
         // ---- sweep 1 of the row after this one, so that one barrier per row serves both
         // (a row three or more further on has not been asked for yet: its sweep waits until this row is done)
         const int kn = next_active(k + 1);
@@ -183,7 +184,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             for (int j = 0; j < JV; ++j) {
                 if (FULL || j < nj) {
                     float2 c[NPV];
-                    V::pairs(stage_vec(stage, tid + j * kQThreads), c);
+                    V::pairs(stage_vec(stage, tid + j * NT), c);
 #pragma unroll
                     for (int q = 0; q < NPV; ++q) {
                         const float2 d = __ffma2_rn(c[q], L2, nm2);
@@ -204,7 +205,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             // again with the product of such a code taken as 0.  A real NaN still shows in the sum of exponentials.
             ts = 0.f;
             for (int j = 0; j < nj; ++j) {
-                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * NT) * 16);
 #pragma unroll
                 for (int q = 0; q < VEC; ++q) {
                     const float d = fmaf(Elem<T>::widen(v[q]), kLog2e, -m2);
@@ -231,10 +232,10 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
                 // the thread's lowest index holding the maximum competes for the arg-max
                 int best = INT_MAX;
                 for (int j = nj - 1; j >= 0; --j) {
-                    const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+                    const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * NT) * 16);
 #pragma unroll
                     for (int q = VEC - 1; q >= 0; --q)
-                        if (Elem<T>::widen(v[q]) == m) best = (tid + j * kQThreads) * VEC + q;
+                        if (Elem<T>::widen(v[q]) == m) best = (tid + j * NT) * VEC + q;
                 }
                 if (best != INT_MAX) atomicMin(&sh.argmin[par], best);
             }
@@ -244,14 +245,14 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             if ((lane & 15) == 0) pk.wsum[warp][lane >> 2] = zt;
         }
         __syncwarp();
-        named_bar_sync(kBarRow, kQThreads);
+        named_bar_sync(kBarRow, NT);
         if (sh.abort) {
             aborted = true;
             break;
         }
-        float z = pk.wsum[lane & (kQWarps - 1)][0];
+        float z = pk.wsum[lane & (NW - 1)][0];
 #pragma unroll
-        for (int ofs = 8; ofs > 0; ofs >>= 1) z += __shfl_xor_sync(0xffffffffu, z, ofs);
+        for (int ofs = NW / 2; ofs > 0; ofs >>= 1) z += __shfl_xor_sync(0xffffffffu, z, ofs);
         const int nmax = sh.nmax[it & 3];
         z = fmaf((float)nmax, e0, z);
         const float rho = pk.rho;
@@ -261,10 +262,10 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             // an unusable row (NaN / +inf logit, no finite logit): classify it from the landed bytes
             // exactly as the row-status bits are defined
             if (tid == 0) sh.bad_nan = sh.bad_finite = 0;
-            named_bar_sync(kBarRow, kQThreads);
+            named_bar_sync(kBarRow, NT);
             int has_nan = 0, has_finite = 0;
             for (int j = 0; j < nj; ++j) {
-                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * NT) * 16);
 #pragma unroll
                 for (int q = 0; q < VEC; ++q) {
                     const float c = Elem<T>::widen(v[q]);
@@ -274,7 +275,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             }
             if (has_nan) sh.bad_nan = 1;
             if (has_finite) sh.bad_finite = 1;
-            named_bar_sync(kBarRow, kQThreads);
+            named_bar_sync(kBarRow, NT);
             if (sh.bad_nan) status |= CIAR_ROW_NAN;
             if (!sh.bad_finite) status |= CIAR_ROW_NO_FINITE;
             if (!status) status = CIAR_ROW_NAN;  // sums overflowed without any single bad logit
@@ -351,7 +352,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             float ps[5] = { 0.f, 0.f, 0.f, 0.f, 0.f };
 #pragma unroll 1
             for (int j = 0; j < nj; ++j) {
-                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kQThreads) * 16);
+                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * NT) * 16);
                 float c[VEC];
                 Elem<T>::load(v, c);
 #pragma unroll
@@ -372,7 +373,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
             r0 = warp_sum_pair(ps[0], ps[1], lane);
             r1 = warp_sum_pair(ps[2], ps[3], lane);
             r2 = warp_sum_f(ps[4]);
-            named_bar_sync(kBarRow, kQThreads);
+            named_bar_sync(kBarRow, NT);
             if (tid == 0) {
                 fence_proxy_async_smem();
                 issue(k + kQStages);
@@ -390,7 +391,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
         // A row parked before this one may have listed more codes than its slot holds; the rest sits in the
         // shared buffer of its parity, which the row after this one reuses: finish the parked rows now.
         const bool long_pending = filled > 0 && sh.park[filled - 1].nlist > kParkList;
-        if (++filled == kPark || long_pending) {
+        if (++filled == NW || long_pending) {
             finish_parked(filled);
             filled = 0;
         }
@@ -399,7 +400,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
         if (MAPPED && k >= 0 && !ahead) {  // the next row's first sweep could not run ahead: it runs here, with a barrier of its own
             first_sweep(k, it);
             __syncwarp();
-            named_bar_sync(kBarRow, kQThreads);
+            named_bar_sync(kBarRow, NT);
             if (sh.abort) aborted = true;
         }
     }
@@ -417,35 +418,35 @@ __global__ void __launch_bounds__(kQThreads, MINB) quantify_stream_kernel(const 
     }
 }
 
-template <typename T, int JV, int MINB, bool FULL, bool MAPPED>
+template <typename T, int NT, int JV, int MINB, bool FULL, bool MAPPED>
 cudaError_t launch_one(const QuantifyArgs &a, cudaStream_t stream)
 {
-    constexpr size_t smem = (size_t)kQStages * kQThreads * JV * 16 + sizeof(QShared);
+    constexpr size_t smem = (size_t)kQStages * NT * JV * 16 + sizeof(QShared);
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        err = cudaFuncSetAttribute(quantify_stream_kernel<T, JV, MINB, FULL, MAPPED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        err = cudaFuncSetAttribute(quantify_stream_kernel<T, NT, JV, MINB, FULL, MAPPED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)smem);
         if (err != cudaSuccess) return err;
         configured[dev] = true;
     }
     const int64_t cap = (int64_t)sm_count() * MINB;
     const unsigned grid = (unsigned)(a.rows < cap ? a.rows : cap);
-    quantify_stream_kernel<T, JV, MINB, FULL, MAPPED><<<grid, kQThreads, smem, stream>>>(a);
+    quantify_stream_kernel<T, NT, JV, MINB, FULL, MAPPED><<<grid, NT, smem, stream>>>(a);
     count_launch();
     return cudaGetLastError();
 }
 
-template <typename T, int JV, int MINB>
+template <typename T, int NT, int JV, int MINB>
 cudaError_t launch_jv(const QuantifyArgs &a, cudaStream_t stream)
 {
     const int nvec = a.n / Elem<T>::kVec;
     const bool mapped = a.rm.pos != nullptr;
-    if (nvec == kQThreads * JV) return mapped ? launch_one<T, JV, MINB, true, true>(a, stream) : launch_one<T, JV, MINB, true, false>(a, stream);
-    return mapped ? launch_one<T, JV, MINB, false, true>(a, stream) : launch_one<T, JV, MINB, false, false>(a, stream);
+    if (nvec == NT * JV) return mapped ? launch_one<T, NT, JV, MINB, true, true>(a, stream) : launch_one<T, NT, JV, MINB, true, false>(a, stream);
+    return mapped ? launch_one<T, NT, JV, MINB, false, true>(a, stream) : launch_one<T, NT, JV, MINB, false, false>(a, stream);
 }
 
 }  // namespace
@@ -463,13 +464,15 @@ cudaError_t launch_quantify_stream(const QuantifyArgs &a, int dtype, cudaStream_
 {
     if (a.rows == 0) return cudaSuccess;
     if (dtype == CIAR_F32) {
-        if (a.n <= 4096) return launch_jv<float, 2, 2>(a, stream);
-        if (a.n <= 8192) return launch_jv<float, 4, 2>(a, stream);
-        return launch_jv<float, 8, 1>(a, stream);
+        if (a.n <= 4096) return launch_jv<float, 512, 2, 2>(a, stream);
+        if (a.n <= 8192) return launch_jv<float, 512, 4, 2>(a, stream);
+        return launch_jv<float, 512, 8, 1>(a, stream);
     }
-    if (a.n <= 4096) return launch_jv<__nv_bfloat16, 1, 2>(a, stream);
-    if (a.n <= 8192) return launch_jv<__nv_bfloat16, 2, 2>(a, stream);
-    return launch_jv<__nv_bfloat16, 4, 2>(a, stream);
+    // Short rows go to CTAs of 256 threads, three per SM: a thread then still owns 16 or 32 codes of a row, over
+    // which the per-row work (reductions, barrier, parking) is spread.
+    if (a.n <= 4096) return launch_jv<__nv_bfloat16, 256, 2, 3>(a, stream);
+    if (a.n <= 8192) return launch_jv<__nv_bfloat16, 256, 4, 3>(a, stream);
+    return launch_jv<__nv_bfloat16, 512, 4, 2>(a, stream);
 }
 
 }  // namespace ciar

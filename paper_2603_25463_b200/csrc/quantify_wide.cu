@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(kWThreads, 1) quantify_wide_kernel(const __gri
                 __syncwarp();
                 list = sh.list;
             }
-            finish_row(a, p, list, lane);
+            finish_row(a, p, list, lane, kQWarps);
         }
         __syncthreads();
     };
