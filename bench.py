@@ -195,8 +195,6 @@ def run_ours(args):
     barrier(world)
     clocks = sampler.stop()
     launches = ciar.launch_count() - launches0
-    if graph is not None:
-        launches = steps * launches_per_step  # replays do not pass through the library's counter
     total_ms = max_over_ranks(t_start.elapsed_time(t_end), world)
     q_ms = float(np.mean([ev[k][0].elapsed_time(ev[k][1]) for k in range(K)]))
     v_ms = float(np.mean([ev[k][1].elapsed_time(ev[k][2]) for k in range(K)]))
