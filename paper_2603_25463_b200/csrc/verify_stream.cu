@@ -237,8 +237,8 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
     int k = 0, filled = 0;
     bool aborted = false;
     // Waits for this CTA's kk-th row to land and takes the maximum over it (sweep 1): each warp's maximum goes
-    // to the slot of the row's parity.  Thread 0 also clears the row's count of maxima.
-    auto first_sweep = [&](int kk) {
+    // to the slot of the row's parity.  Thread 0 also clears the row's count of maxima.  Returns the thread's maximum.
+    auto first_sweep = [&](int kk) -> float {
         const int s = kk % kVStages;
         const unsigned char *stage = smem + (size_t)s * kStageBytes;
         if (mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kWaitCycles)) phases ^= 1u << s;
@@ -247,13 +247,16 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
 #pragma unroll
         for (int j = 0; j < JV; ++j)
             if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * kVThreads));
-        const float wm = warp_redux_max(V::max_value(mx));
+        const float tmax = V::max_value(mx);
+        const float wm = warp_redux_max(tmax);
         if (lane == 0) sh.wmax[kk & 1][warp] = wm;
         if (tid == 0) sh.nmax[kk & 3] = 0;
+        return tmax;
     };
     const int mine = blockIdx.x < total ? (total - 1 - (int)blockIdx.x) / stride + 1 : 0;  // rows this CTA walks
+    float tm = 0.f;  // this thread's maximum of the row being summed
     if (mine > 0) {
-        first_sweep(0);
+        tm = first_sweep(0);
         __syncwarp();
         __syncthreads();
         if (sh.abort) aborted = true;
@@ -265,7 +268,8 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
         const int par = k & 1;
         const unsigned char *stage = smem + (size_t)s * kStageBytes;
         const float m = warp_redux_max(sh.wmax[par][lane & (kVWarps - 1)]);
-        if (k + 1 < mine) first_sweep(k + 1);
+        float tmn = 0.f;
+        if (k + 1 < mine) tmn = first_sweep(k + 1);
         // sweep 2: sum of exponentials; terms equal to the maximum's are counted, not summed
         const float m2 = m * kLog2e;
         const float e0 = ex2_approx(fmaf(m, kLog2e, -m2));
@@ -286,19 +290,24 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
             }
         }
         float zs = z2.x + z2.y;
-        if (sh.wmax[par][warp] == m) {  // a warp holding a maximum redoes its sums without the maxima (kept exactly, as a count)
+        // A thread holding a maximum has its sum formed again without the maxima (kept exactly, as a count): a term
+        // near 1 would cost the small terms their low bits.  The whole warp does it for the thread, a code per lane.
+        for (unsigned holders = __ballot_sync(0xffffffffu, tm == m); holders != 0; holders &= holders - 1) {
+            const int h = __ffs((int)holders) - 1;
+            const int htid = (tid & ~31) + h;
+            const int hn = (FULL ? JV : __shfl_sync(0xffffffffu, nj, h)) * VEC;  // the thread's codes
             float zz = 0.f;
             int cnt = 0;
-            for (int j = 0; j < nj; ++j) {
-                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * kVThreads) * 16);
-#pragma unroll
-                for (int q = 0; q < VEC; ++q) {
-                    const float ev = ex2_approx(fmaf(Elem<T>::widen(v[q]), kLog2e, -m2));
-                    if (ev == e0) ++cnt; else zz += ev;
-                }
+            for (int i = lane; i < hn; i += 32) {
+                const T *v = reinterpret_cast<const T *>(stage + (size_t)(htid + (i / VEC) * kVThreads) * 16);
+                const float ev = ex2_approx(fmaf(Elem<T>::widen(v[i % VEC]), kLog2e, -m2));
+                if (ev == e0) ++cnt; else zz += ev;
             }
-            zs = zz;
-            if (cnt > 0) atomicAdd(&sh.nmax[k & 3], cnt);
+            zz = warp_sum_f(zz);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+            if (lane == h) zs = zz;
+            if (lane == 0 && cnt > 0) atomicAdd(&sh.nmax[k & 3], cnt);
         }
         const float wz = warp_sum_f(zs);
         VParked &pk = sh.park[filled];
@@ -320,6 +329,7 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
             finish_parked(filled);
             filled = 0;
         }
+        tm = tmn;
     }
     if (filled > 0) finish_parked(filled);
     if (aborted && tid == 0) {
