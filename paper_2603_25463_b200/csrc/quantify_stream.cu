@@ -215,29 +215,37 @@ __global__ void __launch_bounds__(NT, MINB) quantify_stream_kernel(const __grid_
         }
         const float e0 = ex2_approx(fmaf(m, kLog2e, -m2));  // the exponential every maximum got
         if (sh.wmax[par][warp] == m) {
-            // This warp owns a maximum.  A term near 1 would cost the small terms their low bits, so its threads
-            // form their partial sums again without the terms equal to e0; they come back exactly, as a count.
-            float zz = 0.f;
-            int cnt = 0;
+            // This warp owns a maximum.  A term near 1 would cost the small terms their low bits, so the sum of a
+            // thread that holds one is formed again without the terms equal to e0 (they come back exactly, as a
+            // count), by the whole warp, a code per lane; the lowest such code competes for the arg-max.
+            typename V::Max mx = V::max_init();
 #pragma unroll
-            for (int i = 0; i < NP; ++i) {
-                if (FULL || i / NPV < nj) {
-                    if (e[i].x == e0) ++cnt; else zz += e[i].x;
-                    if (e[i].y == e0) ++cnt; else zz += e[i].y;
+            for (int j = 0; j < JV; ++j)
+                if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * NT));
+            for (unsigned holders = __ballot_sync(0xffffffffu, V::max_value(mx) == m); holders != 0; holders &= holders - 1) {
+                const int h = __ffs((int)holders) - 1;
+                const int htid = (tid & ~31) + h;
+                const int hn = (FULL ? JV : __shfl_sync(0xffffffffu, nj, h)) * VEC;  // the thread's codes
+                float zz = 0.f;
+                int cnt = 0, first = INT_MAX;
+                for (int i = lane; i < hn; i += 32) {
+                    const int vi = htid + (i / VEC) * NT;
+                    const float c = Elem<T>::widen(reinterpret_cast<const T *>(stage + (size_t)vi * 16)[i % VEC]);
+                    const float ev = ex2_approx(fmaf(c, kLog2e, -m2));
+                    if (ev == e0) ++cnt; else zz += ev;
+                    if (c == m) first = min(first, vi * VEC + i % VEC);
                 }
-            }
-            zs = zz;
-            if (cnt > 0) {
-                atomicAdd(&sh.nmax[it & 3], cnt);
-                // the thread's lowest index holding the maximum competes for the arg-max
-                int best = INT_MAX;
-                for (int j = nj - 1; j >= 0; --j) {
-                    const T *v = reinterpret_cast<const T *>(stage + (size_t)(tid + j * NT) * 16);
+                zz = warp_sum_f(zz);
 #pragma unroll
-                    for (int q = VEC - 1; q >= 0; --q)
-                        if (Elem<T>::widen(v[q]) == m) best = (tid + j * NT) * VEC + q;
+                for (int o = 16; o > 0; o >>= 1) {
+                    cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+                    first = min(first, __shfl_xor_sync(0xffffffffu, first, o));
                 }
-                if (best != INT_MAX) atomicMin(&sh.argmin[par], best);
+                if (lane == h) zs = zz;
+                if (lane == 0) {
+                    if (cnt > 0) atomicAdd(&sh.nmax[it & 3], cnt);
+                    if (first != INT_MAX) atomicMin(&sh.argmin[par], first);
+                }
             }
         }
         {
