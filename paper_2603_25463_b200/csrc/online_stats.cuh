@@ -37,7 +37,8 @@ __device__ __forceinline__ void online_sweep(OnlineStats &st, const unsigned cha
 #pragma unroll
     for (int j = 0; j < JV; ++j)
         if (WHOLE || j < nj) mx = V::fold_max(mx, stage_vec(stage, tg + j * NT));
-    const float wmc = warp_redux_max(V::max_value(mx));
+    const float tmax = V::max_value(mx);
+    const float wmc = warp_redux_max(tmax);
     if (wmc > st.m_w) {  // the maximum moves: what was summed so far is rescaled to it (in double)
         if (st.m_w > -INFINITY) {
             const float m2o = st.m_w * kLog2e;
@@ -84,20 +85,31 @@ __device__ __forceinline__ void online_sweep(OnlineStats &st, const unsigned cha
             }
         }
         if (wmc == st.m_w) {
-            // This chunk holds codes equal to the warp's maximum: the sum is formed again without them; they are counted.
+            // This chunk holds codes equal to the warp's maximum.  The sum of a thread that holds one is formed again
+            // without them, by the whole warp, a code per lane; they are counted instead.
             const float e0w = ex2_approx(fmaf(st.m_w, kLog2e, -m2w));
-            float zz = 0.f;
-            for (int j = 0; j < nj; ++j) {
-                const T *v = reinterpret_cast<const T *>(stage + (size_t)(tg + j * NT) * 16);
+            const int lane = threadIdx.x & 31;
+            for (unsigned holders = __ballot_sync(0xffffffffu, tmax == st.m_w); holders != 0; holders &= holders - 1) {
+                const int h = __ffs((int)holders) - 1;
+                const int htg = (tg & ~31) + h;
+                const int hn = (WHOLE ? JV : __shfl_sync(0xffffffffu, nj, h)) * VEC;  // the thread's codes in this chunk
+                float zz = 0.f;
+                int cnt = 0;
+                for (int i = lane; i < hn; i += 32) {
+                    const T *v = reinterpret_cast<const T *>(stage + (size_t)(htg + (i / VEC) * NT) * 16);
+                    const float ev = ex2_approx(fmaf(Elem<T>::widen(v[i % VEC]), kLog2e, -m2w));
+                    if (ev == e0w) ++cnt; else zz += ev;
+                }
+                zz = warp_sum_f(zz);
 #pragma unroll
-                for (int q = 0; q < VEC; ++q) {
-                    const float ev = ex2_approx(fmaf(Elem<T>::widen(v[q]), kLog2e, -m2w));
-                    if (ev == e0w) ++st.cnt; else zz += ev;
+                for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+                if (lane == h) {
+                    zs = zz;
+                    st.cnt += cnt;
                 }
             }
-            zs = zz;
         }
-    st.zd += (double)zs;
+        st.zd += (double)zs;
         if (WITH_T) st.td += (double)ts;
     }
 }
