@@ -199,11 +199,14 @@ __device__ __forceinline__ void row_stats(const RowView<T> &rv, float *fscratch,
     st.m = m;
     const float m2 = m * kLog2e;
     st.m2 = m2;
-    double acc[2] = { 0.0, 0.0 };
-    // fp32 partial sums over short runs, folded into double so that long rows lose nothing
+    double acc[3] = { 0.0, 0.0, 0.0 };
+    // fp32 partial sums over short runs, folded into double so that long rows lose nothing.  Codes equal to the
+    // maximum are counted, not summed: their term 2^off is put in exactly below (an approximate exponential
+    // of a term near 1 would leave its error, ~1e-7, in ln z of a row that is all but one-hot).
     int32_t vi = rv.vec_begin + threadIdx.x;
     while (vi < rv.vec_end) {
         float z = 0.f, t = 0.f;
+        int cnt = 0;
 #pragma unroll 4
         for (int it = 0; it < 8 && vi < rv.vec_end; ++it, vi += kThreads) {
             float v[V];
@@ -212,18 +215,27 @@ __device__ __forceinline__ void row_stats(const RowView<T> &rv, float *fscratch,
             for (int k = 0; k < V; ++k) {
                 const float d = fmaf(v[k], kLog2e, -m2);
                 const float e = ex2_approx(d);  // NaN logits stay NaN here and poison z on purpose
-                z += e;
-                t = fmaf(e, fmaxf(d, kNegHuge), t);  // -inf logit: e = 0 and 0 * (-1e30) = 0
+                if (v[k] == m) {
+                    ++cnt;
+                } else {
+                    z += e;
+                    t = fmaf(e, fmaxf(d, kNegHuge), t);  // -inf logit: e = 0 and 0 * (-1e30) = 0
+                }
             }
         }
         acc[0] += (double)z;
         acc[1] += (double)t;
+        acc[2] += (double)cnt;
     }
-    block_sum<2>(acc, dscratch);
-    st.z_raw = acc[0];
+    block_sum<3>(acc, dscratch);
     // exponent actually used: c*log2e_f - m2 = (c - m)*log2e_f + off, off = m*log2e_f - m2, so
-    // z_raw = 2^off * z and t_raw = 2^off * (t + off * z)
+    // z_raw = 2^off * z and t_raw = 2^off * (t + off * z); a maximum code's own terms are 2^off and 2^off * off
+    // (a +inf maximum makes off NaN, which marks the row as before)
     const double off = (double)m * (double)kLog2e - (double)m2;
+    const double scale = exp2(off);
+    acc[0] += acc[2] * scale;
+    acc[1] += acc[2] * scale * off;
+    st.z_raw = acc[0];
     const double unscale = exp2(-off);
     st.z = acc[0] * unscale;
     st.t = acc[1] * unscale - off * st.z;

@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyArgs a)
 {
     constexpr int V = Elem<T>::kVec;
     __shared__ float fs[kWarps];
-    __shared__ double ds[2 * kWarps];
+    __shared__ double ds[3 * kWarps];
     __shared__ double scan_warp[kWarps];
     __shared__ double sh_d[4];
     __shared__ int sh_i[4];  // 0: accept bit, 2..3: scratch of the resampler

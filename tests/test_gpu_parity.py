@@ -86,17 +86,18 @@ def test_quantify_radius_extremes_and_closed_forms(ciar, r):
 
 def test_quantify_degenerate_rows(ciar):
     v = 520
+    g = torch.Generator().manual_seed(520)
     rows = []
     one_hot = torch.full((v,), float("-inf")); one_hot[17] = 2.5; rows.append(one_hot)
     rows.append(torch.full((v,), -0.75))  # constant row: Sigma = 0
     near = torch.full((v,), -30.0); near[100] = 20.0; rows.append(near)  # p_max = 1 - 5e-20
     two = torch.full((v,), float("-inf")); two[3] = 1.0; two[400] = 1.0; rows.append(two)
     ties = torch.zeros(v); ties[40:44] = 5.0; rows.append(ties)  # arg-max tie -> lowest index
-    nan_row = torch.randn(v); nan_row[7] = float("nan"); rows.append(nan_row)
+    nan_row = torch.randn(v, generator=g); nan_row[7] = float("nan"); rows.append(nan_row)
     rows.append(torch.full((v,), float("-inf")))  # no finite code
-    inf_row = torch.randn(v); inf_row[9] = float("inf"); rows.append(inf_row)
-    big = torch.randn(v) * 1e4; rows.append(big)  # huge dynamic range
-    flat_small = torch.randn(v) * 1e-3; rows.append(flat_small)  # nearly uniform widths (low CV)
+    inf_row = torch.randn(v, generator=g); inf_row[9] = float("inf"); rows.append(inf_row)
+    big = torch.randn(v, generator=g) * 1e4; rows.append(big)  # huge dynamic range
+    flat_small = torch.randn(v, generator=g) * 1e-3; rows.append(flat_small)  # nearly uniform widths (low CV)
     logits = torch.stack(rows)
     for dtype in (torch.float32, torch.bfloat16):
         for r in (0.0, 0.3, 2.0):
