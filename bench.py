@@ -123,12 +123,16 @@ def max_over_ranks(x: float, world: int) -> float:
 class Step:
     """The hot path on one resident batch: quantify -> verify through the C ABI binding."""
 
-    def __init__(self, ciar, wl, inp):
+    def __init__(self, ciar, wl, inp, per_code=False):
         self.ciar, self.wl = ciar, wl
         dev = inp.draft.device
         self.draft, self.target = inp.draft, inp.target
         self.tokens, self.ua, self.ur = inp.tokens, inp.u_accept, inp.u_resample
-        self.params = ciar.IntervalParams(radius_mode=ciar.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
+        if per_code:  # one raw radius per code, as the interval head emits it (Softplus applied on the device)
+            self.params = ciar.IntervalParams(radius_mode=ciar.RADIUS_PER_CODE, radius=inp.radius_code, radius_is_raw=True,
+                                              tau=wl.tau)
+        else:
+            self.params = ciar.IntervalParams(radius_mode=ciar.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
         rows = inp.draft.shape[0]
         self.rows = rows
         self.qout = ciar.QuantifyOut.allocate(rows, dev)
@@ -166,8 +170,9 @@ def run_ours(args):
     if args.images:
         wl = wl.scaled(images=args.images)  # a smaller batch of the same recipe (profiler captures)
     wl = ciar_dist.rank_workload(wl, rank)  # every rank draws its own batch (weak scaling)
-    inp = synth.make_inputs(wl, device=dev)
-    step = Step(ciar, wl, inp)
+    per_code = args.radius == "per_code"
+    inp = synth.make_inputs(wl, device=dev, per_code_radius=per_code)
+    step = Step(ciar, wl, inp, per_code)
     rows = step.rows
     row_bytes = wl.n_valid * wl.elem_bytes
 
@@ -205,7 +210,8 @@ def run_ours(args):
     e2e = None
     if not args.no_e2e:
         hd, ht = inp.draft.cpu().pin_memory(), inp.target.cpu().pin_memory()
-        htok, hua, hur, hrad = (x.cpu().pin_memory() for x in (inp.tokens, inp.u_accept, inp.u_resample, inp.radius_row))
+        htok, hua, hur, hrad = (x.cpu().pin_memory() for x in (inp.tokens, inp.u_accept, inp.u_resample,
+                                                               inp.radius_code if per_code else inp.radius_row))
         res_dev = [step.qout.flag, step.qout.score, step.vout.accept, step.vout.accepted_len, step.vout.resampled_token,
                    step.vout.first_flag]
         res_host = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in res_dev]
@@ -237,16 +243,18 @@ def run_ours(args):
     if rank != 0:
         return
     peak, peak_kind = measured_peak()
-    q_bytes = rows * row_bytes + rows * 48
+    q_bytes = rows * row_bytes * (2 if per_code else 1) + rows * 48  # a per-code radius row is as wide as its logit row
     v_bytes = sent * row_bytes + resampled * 2 * row_bytes + rows * 16 + (rows // wl.window) * 16
     q_gbs = q_bytes / (q_ms * 1e-3) / 1e9
     v_gbs = v_bytes / (v_ms * 1e-3) / 1e9
     wide = wl.n_valid > 16384  # rows that do not fit on chip take the two-pass / chunked kernels
     q_name = "quantify_wide_kernel" if wide else "quantify_stream_kernel"
+    if per_code:
+        q_name = "quantify_kernel"
     v_name = "verify_plan+accept_wide+window" if wide else "verify_plan+accept+window"
     dominant = q_name if q_ms >= v_ms else v_name
     dom_gbs = q_gbs if q_ms >= v_ms else v_gbs
-    traffic = load_traffic(dominant, args.workload)
+    traffic = None if per_code else load_traffic(dominant, args.workload)
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
                 "frac": dom_gbs / peak, "peak_kind": "of " + peak_kind, "traffic": traffic,
                 "frac_of_nominal_8TBs": dom_gbs / NOMINAL_HBM_GBS,
@@ -263,7 +271,7 @@ def run_ours(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "rows_per_gpu": rows, "vocab": wl.vocab, "valid_codes": wl.n_valid,
-                   "logits": wl.dtype, "window": wl.window, "verify_mode": "anchored", "radius": "per_row",
+                   "logits": wl.dtype, "window": wl.window, "verify_mode": "anchored", "radius": args.radius,
                    "tau": wl.tau, "l2": "inputs (%.0f MB) larger than L2; no flush" % (2 * rows * row_bytes / 1e6)},
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
@@ -390,7 +398,7 @@ def run_decode(args):
         "steps": steps, "warmup": 1, "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "decode", "requests_per_gpu": req, "seq_len": seq, "vocab": wl.vocab, "logits": wl.dtype,
-                   "window": wl.window, "verify_mode": "anchored", "radius": "per_row", "tau": wl.tau,
+                   "window": wl.window, "verify_mode": "anchored", "radius": args.radius, "tau": wl.tau,
                    "launch": "cuda graph replay" if graph is not None else "direct",
                    "l2": "pools of %.1f GB, rows touched once" % (2 * req * seq * wl.vocab * wl.elem_bytes / 1e9)},
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
@@ -455,6 +463,8 @@ def main():
                     help="images of the workload (default: the workload's own); a smaller batch for profiler captures")
     ap.add_argument("--decode-graph", action=argparse.BooleanOptionalAction, default=True,
                     help="decode workload: replay each step from a CUDA graph (default) or launch it directly")
+    ap.add_argument("--radius", default="per_row", choices=["per_row", "per_code"],
+                    help="interval radius: one per row (default) or one raw value per code, a tensor as large as the logits")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
