@@ -250,7 +250,7 @@ def run_ours(args):
     wide = wl.n_valid > 16384  # rows that do not fit on chip take the two-pass / chunked kernels
     q_name = "quantify_wide_kernel" if wide else "quantify_stream_kernel"
     if per_code:
-        q_name = "quantify_kernel"
+        q_name = "quantify_percode_kernel"
     v_name = "verify_plan+accept_wide+window" if wide else "verify_plan+accept+window"
     dominant = q_name if q_ms >= v_ms else v_name
     dom_gbs = q_gbs if q_ms >= v_ms else v_gbs

@@ -61,6 +61,9 @@ cudaError_t launch_quantify_stream(const QuantifyArgs &a, int dtype, cudaStream_
 // The streaming quantifier for rows wider than that one takes (two passes over a row, chunk by chunk).
 bool quantify_wide_eligible(const QuantifyArgs &a, int dtype);
 cudaError_t launch_quantify_wide(const QuantifyArgs &a, int dtype, cudaStream_t stream);
+// The streaming quantifier for one radius per code (logits and radii through the same TMA ring).
+bool quantify_percode_eligible(const QuantifyArgs &a, int dtype);
+cudaError_t launch_quantify_percode(const QuantifyArgs &a, int dtype, cudaStream_t stream);
 cudaError_t launch_verify(const VerifyArgs &a, int dtype, cudaStream_t stream);
 // The streaming (plan, TMA-ring accept sweep, per-window finish) verifier and the test that says whether it covers a call.
 bool verify_stream_eligible(const VerifyArgs &a, int dtype);

@@ -251,6 +251,7 @@ cudaError_t launch_quantify(const QuantifyArgs &a, int dtype, cudaStream_t strea
     if (a.rows == 0) return cudaSuccess;
     if (quantify_stream_eligible(a, dtype)) return launch_quantify_stream(a, dtype, stream);
     if (quantify_wide_eligible(a, dtype)) return launch_quantify_wide(a, dtype, stream);
+    if (quantify_percode_eligible(a, dtype)) return launch_quantify_percode(a, dtype, stream);
     const int64_t cap = (int64_t)sm_count() * 16;
     const unsigned grid = (unsigned)(a.rows < cap ? a.rows : cap);
     const bool per_code = a.radius_mode == CIAR_RADIUS_PER_CODE;

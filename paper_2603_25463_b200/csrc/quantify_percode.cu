@@ -1,0 +1,517 @@
+// Streaming quantifier for rows with one interval radius per code (the form in which the interval head emits it):
+// a row's logits AND its radii arrive together through a ring of shared-memory stages filled by bulk (TMA) copies,
+// so both tensors are read from HBM exactly once.
+//
+// One persistent CTA of 32 warps per SM walks rows blockIdx.x, blockIdx.x + gridDim.x, ...; thread 0 issues the two
+// copies of a row three rows ahead.  A landed row is swept three times from shared memory: the maximum; one
+// exponential per code (kept in registers, 16 per thread) with the softmax and entropy sums; then both InterFuse
+// bounds of every code from its own radius, with the five sums Omega and Sigma are built from.  Each sweep ends in
+// a CTA barrier that publishes the per-warp sums; every thread then holds the row's totals.  A row whose widths are
+// nearly uniform gets a fourth sweep that sums (delta - mu)^2 directly (the moment form would cancel).  The row's
+// totals are parked in shared memory; every 32 rows each warp finishes one parked row (logarithm, square root,
+// flag, stores), so that no single thread's scalar work holds up the CTA row after row.
+#include "quantify_finish.cuh"
+
+namespace ciar {
+
+namespace {
+
+constexpr int kPcThreads = 1024;
+constexpr int kPcWarps = kPcThreads / 32;
+constexpr int kPcStages = 3;
+constexpr int kPcJV = 2;          // 16-byte vectors of a row per thread, at most
+constexpr int kPcRowBytes = 32768;  // widest row of one tensor a stage takes (16384 bf16 / 8192 fp32 codes)
+constexpr int kBarPc = 1;
+
+// A row's totals in double: the softmax sums as computed (relative to m2 = fl(m * log2e)) and the five interval sums.
+struct PcTotals {
+    double z_raw, t_raw, A, B, AA, AB, BB;
+};
+
+// A row whose sweeps are done: what the finishing arithmetic needs.
+struct PcParked {
+    PcTotals tt;
+    double dev;  // sum of (delta - mu)^2 from the fourth sweep, when low_cv
+    long long lr;
+    float m;
+    int first, low_cv;
+};
+// (the totals of a parked row already hold a dominant code's unit)
+
+struct PcShared {
+    unsigned long long full[kPcStages];
+    PcParked park[kPcWarps];
+    float wmax[kPcWarps];
+    float zs[kPcWarps], ts[kPcWarps];  // per-warp sums of the sweeps
+    float sums[5][kPcWarps];
+    float dev[kPcWarps];
+    int cnt, first;  // codes equal to the row maximum, and the lowest of them
+    int abort;
+};
+
+// The per-warp sums of a row joined in double (a warp; every lane gets the totals).  The exponent actually used is
+// c * log2e_f - m2 = (c - m) * log2e_f + off with off = m * log2e_f - m2; a code equal to the maximum, left out of
+// the sweeps' sums, contributes exactly 2^off to z_raw and 2^off off to t_raw.  A dominant code (see the kernel) entered
+// the sums of p^l and p^l^2 less 1.
+__device__ __forceinline__ PcTotals row_totals(const PcShared &sh, int lane, float m, int nmax, int dominant)
+{
+    const double off = (double)m * (double)kLog2e - (double)(m * kLog2e);
+    const double scale = exp2(off);
+    PcTotals t;
+    t.z_raw = warp_sum_d((double)sh.zs[lane]) + (double)nmax * scale;
+    t.t_raw = warp_sum_d((double)sh.ts[lane]) + (double)nmax * scale * off;
+    t.A = warp_sum_d((double)sh.sums[0][lane]);
+    t.B = warp_sum_d((double)sh.sums[1][lane]) + (double)dominant;
+    t.AA = warp_sum_d((double)sh.sums[2][lane]);
+    t.AB = warp_sum_d((double)sh.sums[3][lane]);
+    t.BB = warp_sum_d((double)sh.sums[4][lane]) + (double)dominant;
+    return t;
+}
+
+// The normalisation step's scales and what follows from them: delta_i = k_up d_i + g p^l_i, every term >= 0.
+struct PcScales {
+    double k_up, g, omega, mu;
+};
+
+__device__ __forceinline__ PcScales row_scales(const PcTotals &t, float lo_cap, float hi_cap, double nn)
+{
+    const double S_lo = t.B, S_up = t.A + t.B;
+    double k_lo = 1.0, k_up = 1.0;
+    if (S_lo > 0.0 && (double)lo_cap / S_lo < 1.0) k_lo = (double)lo_cap / S_lo;
+    if (S_up > 0.0 && (double)hi_cap / S_up > 1.0) k_up = (double)hi_cap / S_up;
+    PcScales s;
+    s.k_up = k_up;
+    s.g = k_up - k_lo;
+    s.omega = k_up * t.A + s.g * t.B;
+    s.mu = s.omega / nn;
+    return s;
+}
+
+// Interval constants of one code: a = e^-r, alpha = 1 - a, beta = e^r - 1, bma = e^r - e^-r.
+struct CodeRadius {
+    float a, alpha, beta, bma;
+};
+
+// e^r - 1 for a stored (not raw) radius: a short series below 1/2, the exponential itself above.
+__device__ __forceinline__ float expm1_fast(float r)
+{
+    float s = fmaf(r, 1.0f / 7.0f, 1.0f);
+    s = fmaf(r * (1.0f / 6.0f), s, 1.0f);
+    s = fmaf(r * (1.0f / 5.0f), s, 1.0f);
+    s = fmaf(r * (1.0f / 4.0f), s, 1.0f);
+    s = fmaf(r * (1.0f / 3.0f), s, 1.0f);
+    s = fmaf(r * 0.5f, s, 1.0f);
+    const float big = ex2_approx(r * kLog2e) - 1.0f;
+    return fabsf(r) < 0.5f ? r * s : big;
+}
+
+// RAW: the stored value is rho and r = Softplus(rho) = ln(1 + e^rho), so e^r - 1 = e^rho with no logarithm at all;
+// the clamp r <= r_max becomes beta <= e^r_max - 1.
+template <bool RAW>
+__device__ __forceinline__ CodeRadius code_radius_fast(float rho, float r_max, float beta_max)
+{
+    CodeRadius k;
+    if (RAW) k.beta = fminf(ex2_approx(rho * kLog2e), beta_max);
+    else k.beta = expm1_fast(fminf(rho, r_max));
+    if (!(rho == rho)) k.beta = rho;  // fminf drops a NaN operand: a NaN radius must poison its row
+    k.a = rcp_approx(1.0f + k.beta);
+    k.alpha = k.beta * k.a;
+    k.bma = k.alpha + k.beta;
+    return k;
+}
+
+// One code's raw bounds from its softmax probability p:
+//   p^l = a p / (1 - alpha p),  d = p^u - p^l = p (b - a)(1 - p) / ((1 - alpha p)(1 + beta p)).
+__device__ __forceinline__ void code_bounds(float p, const CodeRadius &k, float &pl, float &d)
+{
+    const float den_l = fmaf(-k.alpha, p, 1.0f);
+    const float den_u = fmaf(k.beta, p, 1.0f);
+    const float q = p * rcp_approx(den_l * den_u);
+    pl = k.a * (q * den_u);
+    d = k.bma * (q * (1.0f - p));
+}
+
+template <typename T, bool RAW>
+__global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const __grid_constant__ QuantifyArgs a)
+{
+    constexpr int NT = kPcThreads, NW = kPcWarps, JV = kPcJV;
+    static_assert(NW == 32, "a lane reads one warp's share");
+    constexpr int VEC = Elem<T>::kVec;
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int nvec = a.n / VEC;
+    const uint32_t row_bytes = (uint32_t)nvec * 16u;
+    const size_t stage_bytes = 2 * (size_t)row_bytes;  // logits, then radii
+    PcShared &sh = *reinterpret_cast<PcShared *>(smem + kPcStages * stage_bytes);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const ciar_quantify_out &o = a.out;
+
+    if (tid == 0) {
+#pragma unroll
+        for (int s = 0; s < kPcStages; ++s) mbar_init(&sh.full[s], 1);
+        sh.abort = 0;
+        sh.cnt = 0;
+        sh.first = INT_MAX;
+        mbar_init_fence();
+    }
+    __syncthreads();
+
+    auto row_of = [&](int k) -> int64_t { return blockIdx.x + (int64_t)k * gridDim.x; };
+    auto issue = [&](int k) {  // thread 0 only
+        const int64_t lr = row_of(k);
+        if (lr < a.rows) {
+            const int s = k % kPcStages;
+            unsigned char *stage = smem + s * stage_bytes;
+            const size_t at = (size_t)(a.vb + lr * a.row_stride);
+            mbar_arrive_expect_tx(&sh.full[s], 2 * row_bytes);
+            bulk_copy_g2s(stage, reinterpret_cast<const T *>(a.logits) + at, row_bytes, &sh.full[s]);
+            bulk_copy_g2s(stage + row_bytes, reinterpret_cast<const T *>(a.radius) + at, row_bytes, &sh.full[s]);
+        }
+    };
+    if (tid == 0) {
+#pragma unroll
+        for (int s = 0; s < kPcStages; ++s) issue(s);
+    }
+
+    const double nn = (double)a.n;
+    // Lane 0 of every warp finishes one parked row.
+    auto finish_parked = [&](int count) {
+        named_bar_sync(kBarPc, NT);
+        if (warp < count && lane == 0) {
+            const PcParked &p = sh.park[warp];
+            const PcTotals &tt = p.tt;
+            const PcScales sc = row_scales(tt, a.lo_cap, a.hi_cap, nn);
+            double var = (sc.k_up * sc.k_up * tt.AA + 2.0 * sc.k_up * sc.g * tt.AB + sc.g * sc.g * tt.BB) / nn - sc.mu * sc.mu;
+            if (p.low_cv) var = p.dev / nn;
+            const float m = p.m;
+            const double off = (double)m * (double)kLog2e - (double)(m * kLog2e);
+            const double unscale = exp2(-off);
+            const double z = tt.z_raw * unscale;
+            const double t = tt.t_raw * unscale - off * z;
+            const double sigma = sqrt(var > 0.0 ? var : 0.0);
+            const double score = sc.omega * sigma;
+            const double lnz = z < 1.5 ? log1p(z - 1.0) : log(z);  // a peaked row: z just above 1
+            const double p_max = 1.0 / z;
+            const double entropy = lnz - kLn2D * t * p_max;
+            const long long lr = p.lr;
+            int fl;
+            switch (a.policy) {
+            case CIAR_POLICY_INTERVAL: fl = score > (double)a.tau; break;
+            case CIAR_POLICY_ENTROPY: fl = entropy > (double)a.tau; break;
+            case CIAR_POLICY_MAXPROB: fl = p_max < (double)a.tau; break;
+            case CIAR_POLICY_RANDOM: fl = a.u_flag[lr] < a.tau; break;
+            default: fl = 1; break;
+            }
+            if (o.row_max) o.row_max[lr] = m;
+            if (o.sum_exp) o.sum_exp[lr] = (float)z;
+            if (o.lse) o.lse[lr] = (float)((double)m + lnz);
+            if (o.p_max) o.p_max[lr] = (float)p_max;
+            if (o.entropy) o.entropy[lr] = (float)entropy;
+            if (o.S_lo) o.S_lo[lr] = (float)tt.B;
+            if (o.S_up) o.S_up[lr] = (float)(tt.A + tt.B);
+            if (o.omega) o.omega[lr] = (float)sc.omega;
+            if (o.sigma) o.sigma[lr] = (float)sigma;
+            if (o.score) o.score[lr] = (float)score;
+            if (o.argmax) o.argmax[lr] = p.first + a.vb;
+            if (o.flag) o.flag[lr] = (uint8_t)fl;
+            if (o.row_status) o.row_status[lr] = 0;
+        }
+    };
+
+    const float beta_max = (float)expm1((double)a.r_max);
+    int filled = 0;
+    const float inv_n = 1.0f / (float)a.n;
+    uint32_t phases = 0;
+    bool aborted = false;
+    int k = 0;
+    for (; row_of(k) < a.rows; ++k) {
+        const int s = k % kPcStages;
+        const unsigned char *stage = smem + s * stage_bytes;
+        const unsigned char *rstage = stage + row_bytes;
+        if (mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kWaitCycles)) phases ^= 1u << s;
+        else sh.abort = 1;
+
+        // ---- sweep 1: the maximum
+        {
+            typename Vec<T>::Max mx = Vec<T>::max_init();
+#pragma unroll
+            for (int j = 0; j < JV; ++j) {
+                const int vi = tid + j * NT;
+                if (vi < nvec) mx = Vec<T>::fold_max(mx, stage_vec(stage, vi));
+            }
+            const float wm = warp_redux_max(Vec<T>::max_value(mx));
+            if (lane == 0) sh.wmax[warp] = wm;
+        }
+        named_bar_sync(kBarPc, NT);
+        if (sh.abort) {
+            aborted = true;
+            break;
+        }
+        const float m = warp_redux_max(sh.wmax[lane]);
+        const float m2 = m * kLog2e;
+
+        // ---- sweep 2: exponentials (kept), their sum and the entropy sum.  Codes whose exponential equals the
+        // maximum's are counted: their terms, 2^off each, enter exactly when the totals are formed.
+        const float e0f = ex2_approx(fmaf(m, kLog2e, -m2));
+        float e[JV * VEC];
+        bool has_max;  // this thread holds a code counted as a maximum
+        {
+            float z = 0.f, t = 0.f;
+            int cnt = 0, first = INT_MAX;
+#pragma unroll
+            for (int j = 0; j < JV; ++j) {
+                const int vi = tid + j * NT;
+                if (vi < nvec) {
+                    float c[VEC];
+                    Elem<T>::load(reinterpret_cast<const T *>(stage + (size_t)vi * 16), c);
+#pragma unroll
+                    for (int q = 0; q < VEC; ++q) {
+                        const float d = fmaf(c[q], kLog2e, -m2);
+                        const float ev = ex2_approx(d);  // a NaN logit poisons z on purpose
+                        e[j * VEC + q] = ev;
+                        if (c[q] == m) first = min(first, vi * VEC + q);
+                        if (ev == e0f) {
+                            ++cnt;
+                        } else {
+                            z += ev;
+                            t = fmaf(ev, fmaxf(d, kNegHuge), t);  // -inf logit: 0 * (-1e30) = 0
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < VEC; ++q) e[j * VEC + q] = 0.f;
+                }
+            }
+            has_max = cnt > 0;
+            const float zt = warp_sum_pair(z, t, lane);  // lanes 0..15: z, lanes 16..31: t
+            if (lane == 0) sh.zs[warp] = zt;
+            if (lane == 16) sh.ts[warp] = zt;
+            if (__any_sync(0xffffffffu, cnt > 0)) {
+#pragma unroll
+                for (int ofs = 16; ofs > 0; ofs >>= 1) {
+                    cnt += __shfl_xor_sync(0xffffffffu, cnt, ofs);
+                    first = min(first, __shfl_xor_sync(0xffffffffu, first, ofs));
+                }
+                if (lane == 0) {
+                    atomicAdd(&sh.cnt, cnt);
+                    atomicMin(&sh.first, first);
+                }
+            }
+        }
+        named_bar_sync(kBarPc, NT);
+        // Every thread needs the row's sum only in float (for 1 / z); the totals in double are formed once, by
+        // warp 0, when it parks the row.  off = m * log2e - m2 is the rounding error of m2; a code equal to the
+        // maximum contributes 2^off.
+        const int nmax = sh.cnt, first = sh.first;
+        const float z_others = warp_sum_f(sh.zs[lane]);
+        const float zf = z_others + (float)nmax * e0f;
+
+        int status = 0;
+        if (m == -INFINITY) status |= CIAR_ROW_NO_FINITE;
+        else if (!(zf < INFINITY) || !(zf > 0.f)) status |= CIAR_ROW_NAN;  // NaN or +inf logit
+        if (status) {
+            // nothing more is read from the stage: hand it to the row three further on
+            named_bar_sync(kBarPc, NT);
+            if (tid == 0) {
+                write_unusable(o, row_of(k), status);
+                sh.cnt = 0;
+                sh.first = INT_MAX;
+                fence_proxy_async_smem();
+                issue(k + kPcStages);
+            }
+            continue;
+        }
+
+        // ---- sweep 3: both bounds of every code from its own radius; the sums of d, p^l, d^2, d p^l, p^l^2
+        const float invz = 1.0f / zf;
+        // A single code that holds more than half of the mass: its p^l, near 1, would cost the sum of the lower bounds
+        // (which decides Omega = 1.01 - S_lo when S_lo < 0.99) its last digits in float.
+        const int dominant = nmax == 1 && e0f * invz > 0.5f;
+        {
+            float sA = 0.f, sB = 0.f, sAA = 0.f, sAB = 0.f, sBB = 0.f;
+            if (!(dominant && has_max)) {
+#pragma unroll
+                for (int j = 0; j < JV; ++j) {
+                    const int vi = tid + j * NT;
+                    if (vi < nvec) {
+                        float rho[VEC];
+                        Elem<T>::load(reinterpret_cast<const T *>(rstage + (size_t)vi * 16), rho);
+#pragma unroll
+                        for (int q = 0; q < VEC; ++q) {
+                            float pl, d;
+                            code_bounds(e[j * VEC + q] * invz, code_radius_fast<RAW>(rho[q], a.r_max, beta_max), pl, d);
+                            sA += d;
+                            sB += pl;
+                            sAA = fmaf(d, d, sAA);
+                            sAB = fmaf(d, pl, sAB);
+                            sBB = fmaf(pl, pl, sBB);
+                        }
+                    }
+                }
+            } else {
+                // The one thread that holds the dominant code.  With s = 1 - x taken from the other codes' sum,
+                // 1 - p^l = s / (a + alpha s) =: q^l keeps its digits, so p^l - 1 = -q^l and p^l^2 - 1 = q^l^2 - 2 q^l
+                // are what this code adds; the units are put back when the totals are formed.
+                const float x_max = e0f * invz, s_max = z_others * invz;
+#pragma unroll
+                for (int j = 0; j < JV; ++j) {
+                    const int vi = tid + j * NT;
+                    if (vi < nvec) {
+                        float rho[VEC];
+                        Elem<T>::load(reinterpret_cast<const T *>(rstage + (size_t)vi * 16), rho);
+#pragma unroll
+                        for (int q = 0; q < VEC; ++q) {
+                            const CodeRadius kr = code_radius_fast<RAW>(rho[q], a.r_max, beta_max);
+                            if (e[j * VEC + q] == e0f) {
+                                const float den_l = fmaf(kr.alpha, s_max, kr.a), den_u = fmaf(kr.beta, x_max, 1.0f);
+                                const float rden = rcp_approx(den_l * den_u);
+                                const float ql = s_max * den_u * rden, d = kr.bma * (x_max * s_max * rden);
+                                sA += d;
+                                sB -= ql;
+                                sAA = fmaf(d, d, sAA);
+                                sAB = fmaf(d, 1.0f - ql, sAB);
+                                sBB += fmaf(ql, ql, -2.0f * ql);
+                            } else {
+                                float pl, d;
+                                code_bounds(e[j * VEC + q] * invz, kr, pl, d);
+                                sA += d;
+                                sB += pl;
+                                sAA = fmaf(d, d, sAA);
+                                sAB = fmaf(d, pl, sAB);
+                                sBB = fmaf(pl, pl, sBB);
+                            }
+                        }
+                    }
+                }
+            }
+            const float r0 = warp_sum_pair(sA, sB, lane), r1 = warp_sum_pair(sAA, sAB, lane), r2 = warp_sum_f(sBB);
+            if (lane == 0) {
+                sh.sums[0][warp] = r0;
+                sh.sums[2][warp] = r1;
+                sh.sums[4][warp] = r2;
+            }
+            if (lane == 16) {
+                sh.sums[1][warp] = r0;
+                sh.sums[3][warp] = r1;
+            }
+        }
+        named_bar_sync(kBarPc, NT);
+        // A look at the totals in float, only to see whether the moment form of the variance is safe for this row
+        // (every thread forms the same values, so the branch below is uniform).
+        bool low_cv;
+        {
+            const float A = warp_sum_f(sh.sums[0][lane]), B = warp_sum_f(sh.sums[1][lane]) + (float)dominant,
+                        AA = warp_sum_f(sh.sums[2][lane]), AB = warp_sum_f(sh.sums[3][lane]),
+                        BB = warp_sum_f(sh.sums[4][lane]) + (float)dominant;
+            const float S_lo = B, S_up = A + B;
+            float k_lo = 1.f, k_up = 1.f;
+            if (S_lo > 0.f && a.lo_cap < S_lo) k_lo = a.lo_cap * rcp_approx(S_lo);
+            if (S_up > 0.f && a.hi_cap > S_up) k_up = a.hi_cap * rcp_approx(S_up);
+            const float g = k_up - k_lo;
+            const float mu = (k_up * A + g * B) * inv_n;
+            const float var = (k_up * k_up * AA + 2.f * k_up * g * AB + g * g * BB) * inv_n - mu * mu;
+            low_cv = !(var >= 0.1f * mu * mu);  // nearly uniform widths: the moment form cancels
+        }
+        double dev_total = 0.0;
+        if (low_cv) {
+            // ---- sweep 4 (rare): sum of (delta_i - mu)^2 with the scales known, from the totals in double
+            const PcTotals tt = row_totals(sh, lane, m, nmax, dominant);
+            const PcScales sc = row_scales(tt, a.lo_cap, a.hi_cap, nn);
+            const float fku = (float)sc.k_up, fg = (float)sc.g, fmu = (float)sc.mu;
+            float sd = 0.f;
+#pragma unroll
+            for (int j = 0; j < JV; ++j) {
+                const int vi = tid + j * NT;
+                if (vi < nvec) {
+                    float rho[VEC];
+                    Elem<T>::load(reinterpret_cast<const T *>(rstage + (size_t)vi * 16), rho);
+#pragma unroll
+                    for (int q = 0; q < VEC; ++q) {
+                        float pl, d;
+                        code_bounds(e[j * VEC + q] * invz, code_radius_fast<RAW>(rho[q], a.r_max, beta_max), pl, d);
+                        const float x = fmaf(fku, d, fg * pl) - fmu;
+                        sd = fmaf(x, x, sd);
+                    }
+                }
+            }
+            sd = warp_sum_f(sd);
+            if (lane == 0) sh.dev[warp] = sd;
+            named_bar_sync(kBarPc, NT);
+            if (warp == 0) dev_total = warp_sum_d((double)sh.dev[lane]);
+        }
+        if (tid == 0) {  // every thread has read the stage for the last time: refill it
+            sh.cnt = 0;
+            sh.first = INT_MAX;
+            fence_proxy_async_smem();
+            issue(k + kPcStages);
+        }
+        if (warp == 0) {  // park the row's totals
+            const PcTotals tt = row_totals(sh, lane, m, nmax, dominant);
+            if (lane == 0) {
+                PcParked &p = sh.park[filled];
+                p.tt = tt;
+                p.dev = dev_total;
+                p.lr = row_of(k);
+                p.m = m;
+                p.first = first;
+                p.low_cv = low_cv;
+            }
+        }
+        if (++filled == NW) {
+            finish_parked(filled);
+            filled = 0;
+        }
+    }
+    if (filled > 0) finish_parked(filled);
+
+    if (aborted && tid == 0) {
+        // A copy never arrived.  Mark this row and the rest of this CTA's rows, then give the copies still in
+        // flight a last bounded chance to land before the CTA leaves.
+        for (int k2 = k; row_of(k2) < a.rows; ++k2) write_unusable(o, row_of(k2), CIAR_ROW_TIMEOUT);
+        for (int s = 0; s < kPcStages; ++s) mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kDrainCycles);
+    }
+}
+
+template <typename T, bool RAW>
+cudaError_t launch_pc(const QuantifyArgs &a, cudaStream_t stream)
+{
+    constexpr size_t smem_max = (size_t)kPcStages * 2 * kPcRowBytes + sizeof(PcShared);
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
+        err = cudaFuncSetAttribute(quantify_percode_kernel<T, RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+        if (err != cudaSuccess) return err;
+        configured[dev] = true;
+    }
+    const size_t row_bytes = (size_t)(a.n / Elem<T>::kVec) * 16;
+    const size_t smem = (size_t)kPcStages * 2 * row_bytes + sizeof(PcShared);
+    const int64_t cap = sm_count();
+    const unsigned grid = (unsigned)(a.rows < cap ? a.rows : cap);
+    quantify_percode_kernel<T, RAW><<<grid, kPcThreads, smem, stream>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool quantify_percode_eligible(const QuantifyArgs &a, int dtype)
+{
+    const int vec = dtype == CIAR_F32 ? 4 : 8;
+    if (a.radius_mode != CIAR_RADIUS_PER_CODE) return false;
+    if (a.rm.pos != nullptr) return false;  // decode row maps stay on the general kernel
+    if (a.out.dense_p || a.out.dense_lo || a.out.dense_up) return false;
+    if (a.vb % vec != 0 || a.n % vec != 0) return false;
+    return a.n >= 2048 && (a.n / vec) * 16 <= kPcRowBytes;
+}
+
+cudaError_t launch_quantify_percode(const QuantifyArgs &a, int dtype, cudaStream_t stream)
+{
+    if (a.rows == 0) return cudaSuccess;
+    if (dtype == CIAR_F32)
+        return a.radius_is_raw ? launch_pc<float, true>(a, stream) : launch_pc<float, false>(a, stream);
+    return a.radius_is_raw ? launch_pc<__nv_bfloat16, true>(a, stream) : launch_pc<__nv_bfloat16, false>(a, stream);
+}
+
+}  // namespace ciar

@@ -76,14 +76,19 @@ def to_ciar_params(p: oracle.IntervalParams, device) -> ciar.IntervalParams:
 
 
 def check_quantify(logits_cpu: torch.Tensor, params: oracle.IntervalParams, valid_begin=0, valid_count=None,
-                   dense=False, device="cuda", logits_dev: Optional[torch.Tensor] = None, threads=0):
-    """Runs both sides on the same rows; returns (oracle result, gpu QuantifyOut, Report)."""
+                   dense=False, device="cuda", logits_dev: Optional[torch.Tensor] = None, threads=0,
+                   radius_dev: Optional[torch.Tensor] = None):
+    """Runs both sides on the same rows; returns (oracle result, gpu QuantifyOut, Report).
+    logits_dev / radius_dev: device tensors to use instead of copies of the CPU ones (strided views)."""
     rows, vocab = logits_cpu.shape
     n = vocab - valid_begin if valid_count is None else valid_count
     ref = oracle.quantify(logits_cpu, params, valid_begin, n, dense=dense, threads=threads)
     ld = logits_cpu.to(device) if logits_dev is None else logits_dev
     out = ciar.QuantifyOut.allocate(rows, device, dense_width=n if dense else 0)
-    ciar.quantify(ld, to_ciar_params(params, device), out, valid_begin, n)
+    gp = to_ciar_params(params, device)
+    if radius_dev is not None:
+        gp.radius = radius_dev
+    ciar.quantify(ld, gp, out, valid_begin, n)
     torch.cuda.synchronize()
     rep = Report(rows=rows)
     for name in Q_FLOAT_FIELDS:

@@ -75,6 +75,68 @@ def test_quantify_radius_modes(ciar, mode, dtype):
     pu.check_quantify(logits, prm, dense=True)
 
 
+@pytest.mark.parametrize("raw", [False, True])
+@pytest.mark.parametrize("dtype,v", [(torch.bfloat16, 2048), (torch.bfloat16, 5000), (torch.bfloat16, 16384),
+                                     (torch.float32, 2052), (torch.float32, 8192)])
+def test_quantify_per_code_radius_streaming_rows(ciar, dtype, v, raw):
+    """Rows of 2048 codes and more with one radius per code (logits and radii streamed together): ordinary
+    rows of several sharpnesses, more rows than a CTA parks, a constant row with constant radii (Sigma = 0),
+    nearly uniform widths, ties of the maximum, -inf stretches, a near one-hot row, unusable rows, radii from
+    tiny to beyond the clamp, stored and raw."""
+    g = torch.Generator().manual_seed(v + int(raw))
+    rows = []
+    for scale in (8.0, 1.0, 3.0, 0.3) * 9:  # 36 ordinary rows
+        rows.append(torch.randn(v, generator=g) * scale)
+    n_ord = len(rows)
+    rows.append(torch.full((v,), -0.75))                        # constant row
+    rows.append(torch.randn(v, generator=g) * 1e-3)             # nearly uniform widths
+    ties = torch.zeros(v); ties[40:44] = 5.0; ties[v - 1] = 5.0; rows.append(ties)
+    holes = torch.randn(v, generator=g); holes[100:1700] = float("-inf"); rows.append(holes)
+    near = torch.full((v,), -30.0); near[v - 9] = 20.0; rows.append(near)
+    nan_row = torch.randn(v, generator=g); nan_row[v - 2] = float("nan"); rows.append(nan_row)
+    rows.append(torch.full((v,), float("-inf")))
+    inf_row = torch.randn(v, generator=g); inf_row[9] = float("inf"); rows.append(inf_row)
+    rows.append(torch.randn(v, generator=g) * 2.0)              # an ordinary row after the unusable ones
+    logits = torch.stack(rows).to(dtype)
+    n = logits.shape[0]
+    if raw:
+        radius = torch.randn(n, v, generator=g) * 1.5 - 1.0     # Softplus -> about 0.03 .. 3
+        radius[1] = -12.0 + torch.randn(v, generator=g)         # tiny radii
+        radius[2] = 6.0 + torch.randn(v, generator=g)           # all beyond the clamp
+    else:
+        radius = torch.rand(n, v, generator=g) * 2.0
+        radius[1] = torch.rand(v, generator=g) * 1e-3
+        radius[2] = 4.0 + torch.rand(v, generator=g)
+        radius[3] = torch.rand(v, generator=g) * 0.6            # both sides of the series / exponential switch
+    radius[n_ord] = 0.4                                         # constant row, constant radius
+    radius[n_ord + 1] = 0.4
+    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_CODE, radius=radius.to(dtype), radius_is_raw=raw,
+                                r_max=2.5, tau=1e-4)
+    ref, out, rep = pu.check_quantify(logits, prm)
+    st = out.row_status.cpu().numpy()
+    assert st[n_ord + 5] == oracle.ROW_NAN and st[n_ord + 6] == oracle.ROW_NO_FINITE and st[n_ord + 7] == oracle.ROW_NAN
+    assert out.argmax.cpu().numpy()[n_ord + 2] == 40
+    assert rep.near_tie_flags <= 1
+
+
+def test_quantify_per_code_radius_streaming_slice(ciar):
+    """The same kernel on a valid slice inside wider rows with a row stride beyond the vocabulary; what lies
+    outside the slice (NaN logits, NaN radii) must never be read."""
+    g = torch.Generator().manual_seed(77)
+    rows, vocab, stride, vb, n = 40, 8192, 8200, 1024, 4096
+    full = torch.full((rows, stride), float("nan"))
+    rfull = torch.full((rows, stride), float("nan"))
+    full[:, vb:vb + n] = torch.randn(rows, n, generator=g) * torch.tensor([8.0, 1.0] * (rows // 2))[:, None]
+    rfull[:, vb:vb + n] = torch.randn(rows, n, generator=g) - 1.0
+    logits = full.to(torch.bfloat16)
+    radius = rfull.to(torch.bfloat16)
+    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_CODE, radius=radius[:, :vocab].contiguous(),
+                                radius_is_raw=True, tau=1e-4)
+    dev = logits.cuda()[:, :vocab]
+    rdev = radius.cuda()[:, :vocab]
+    pu.check_quantify(logits[:, :vocab].contiguous(), prm, valid_begin=vb, valid_count=n, logits_dev=dev, radius_dev=rdev)
+
+
 @pytest.mark.parametrize("r", [0.0, 1e-4, 0.05, 1.0, 5.0, 10.0, 40.0])
 def test_quantify_radius_extremes_and_closed_forms(ciar, r):
     rows, v = 12, 4096
