@@ -87,11 +87,6 @@ __device__ __forceinline__ PcScales row_scales(const PcTotals &t, float lo_cap, 
     return s;
 }
 
-// Interval constants of one code: a = e^-r, alpha = 1 - a, beta = e^r - 1, bma = e^r - e^-r.
-struct CodeRadius {
-    float a, alpha, beta, bma;
-};
-
 // e^r - 1 for a stored (not raw) radius: a short series below 1/2, the exponential itself above.
 __device__ __forceinline__ float expm1_fast(float r)
 {
@@ -105,30 +100,29 @@ __device__ __forceinline__ float expm1_fast(float r)
     return fabsf(r) < 0.5f ? r * s : big;
 }
 
-// RAW: the stored value is rho and r = Softplus(rho) = ln(1 + e^rho), so e^r - 1 = e^rho with no logarithm at all;
-// the clamp r <= r_max becomes beta <= e^r_max - 1.
+// beta = e^r - 1 of one code, r clamped to r_max.  RAW: the stored value is rho and r = Softplus(rho) = ln(1 + e^rho),
+// so beta = e^rho with no logarithm at all, and the clamp becomes beta <= e^r_max - 1.  (The selects keep a NaN
+// radius, which must poison its row.)
 template <bool RAW>
-__device__ __forceinline__ CodeRadius code_radius_fast(float rho, float r_max, float beta_max)
+__device__ __forceinline__ float code_beta(float rho, float r_max, float beta_max)
 {
-    CodeRadius k;
-    if (RAW) k.beta = fminf(ex2_approx(rho * kLog2e), beta_max);
-    else k.beta = expm1_fast(fminf(rho, r_max));
-    if (!(rho == rho)) k.beta = rho;  // fminf drops a NaN operand: a NaN radius must poison its row
-    k.a = rcp_approx(1.0f + k.beta);
-    k.alpha = k.beta * k.a;
-    k.bma = k.alpha + k.beta;
-    return k;
+    if (RAW) {
+        const float u = ex2_approx(rho * kLog2e);
+        return !(u > beta_max) ? u : beta_max;
+    }
+    return expm1_fast(!(rho > r_max) ? rho : r_max);
 }
 
-// One code's raw bounds from its softmax probability p:
-//   p^l = a p / (1 - alpha p),  d = p^u - p^l = p (b - a)(1 - p) / ((1 - alpha p)(1 + beta p)).
-__device__ __forceinline__ void code_bounds(float p, const CodeRadius &k, float &pl, float &d)
+// One code's raw bounds from its exponential e (any common scale), the row's sum z of them and w = z - e:
+//   p^l = e / (z + beta w),   p^u = (1 + beta) e / (z + beta e),
+//   d = p^u - p^l = beta (2 + beta) e w / ((z + beta w)(z + beta e))   -- no cancellation for small radii.
+// (e * rd alone may underflow for a large beta, hence the grouping.)
+__device__ __forceinline__ void code_bounds(float e, float w, float z, float beta, float &pl, float &d)
 {
-    const float den_l = fmaf(-k.alpha, p, 1.0f);
-    const float den_u = fmaf(k.beta, p, 1.0f);
-    const float q = p * rcp_approx(den_l * den_u);
-    pl = k.a * (q * den_u);
-    d = k.bma * (q * (1.0f - p));
+    const float den_l = fmaf(beta, w, z), den_u = fmaf(beta, e, z);
+    const float rd = rcp_approx(den_l * den_u);
+    pl = e * (rd * den_u);
+    d = (fmaf(beta, beta, beta + beta) * rd) * (e * w);
 }
 
 template <typename T, bool RAW>
@@ -256,7 +250,7 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         bool has_max;  // this thread holds a code counted as a maximum
         {
             float z = 0.f, t = 0.f;
-            int cnt = 0, first = INT_MAX;
+            int cnt = 0;
 #pragma unroll
             for (int j = 0; j < JV; ++j) {
                 const int vi = tid + j * NT;
@@ -268,12 +262,11 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                         const float d = fmaf(c[q], kLog2e, -m2);
                         const float ev = ex2_approx(d);  // a NaN logit poisons z on purpose
                         e[j * VEC + q] = ev;
-                        if (c[q] == m) first = min(first, vi * VEC + q);
                         if (ev == e0f) {
                             ++cnt;
                         } else {
                             z += ev;
-                            t = fmaf(ev, fmaxf(d, kNegHuge), t);  // -inf logit: 0 * (-1e30) = 0
+                            t = fmaf(ev, d, t);  // 0 * -inf = NaN for a -inf logit: redone below
                         }
                     }
                 } else {
@@ -282,6 +275,23 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                 }
             }
             has_max = cnt > 0;
+            int first = INT_MAX;
+            if (has_max || !(t == t)) {
+                // A thread that holds a maximum looks for the lowest code equal to it; one whose entropy sum met a
+                // -inf logit (exponential 0, exponent -inf) or a real NaN forms it again with such products taken
+                // as 0 (a real NaN still shows in the sum of exponentials).
+                t = 0.f;
+                for (int vi = tid; vi < nvec; vi += NT) {
+                    const T *cp = reinterpret_cast<const T *>(stage + (size_t)vi * 16);
+#pragma unroll 1
+                    for (int q = 0; q < VEC; ++q) {
+                        const float c = Elem<T>::widen(cp[q]);
+                        const float d = fmaf(c, kLog2e, -m2), ev = ex2_approx(d);
+                        if (c == m) first = min(first, vi * VEC + q);
+                        if (ev != e0f) t = fmaf(ev, fmaxf(d, kNegHuge), t);
+                    }
+                }
+            }
             const float zt = warp_sum_pair(z, t, lane);  // lanes 0..15: z, lanes 16..31: t
             if (lane == 0) sh.zs[warp] = zt;
             if (lane == 16) sh.ts[warp] = zt;
@@ -322,10 +332,9 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         }
 
         // ---- sweep 3: both bounds of every code from its own radius; the sums of d, p^l, d^2, d p^l, p^l^2
-        const float invz = 1.0f / zf;
         // A single code that holds more than half of the mass: its p^l, near 1, would cost the sum of the lower bounds
         // (which decides Omega = 1.01 - S_lo when S_lo < 0.99) its last digits in float.
-        const int dominant = nmax == 1 && e0f * invz > 0.5f;
+        const int dominant = nmax == 1 && e0f > 0.5f * zf;
         {
             float sA = 0.f, sB = 0.f, sAA = 0.f, sAB = 0.f, sBB = 0.f;
             if (!(dominant && has_max)) {
@@ -338,7 +347,8 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
 #pragma unroll
                         for (int q = 0; q < VEC; ++q) {
                             float pl, d;
-                            code_bounds(e[j * VEC + q] * invz, code_radius_fast<RAW>(rho[q], a.r_max, beta_max), pl, d);
+                            const float ev = e[j * VEC + q];
+                            code_bounds(ev, zf - ev, zf, code_beta<RAW>(rho[q], a.r_max, beta_max), pl, d);
                             sA += d;
                             sB += pl;
                             sAA = fmaf(d, d, sAA);
@@ -350,8 +360,8 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
             } else {
                 // The one thread that holds the dominant code.  With s = 1 - x taken from the other codes' sum,
                 // 1 - p^l = s / (a + alpha s) =: q^l keeps its digits, so p^l - 1 = -q^l and p^l^2 - 1 = q^l^2 - 2 q^l
-                // are what this code adds; the units are put back when the totals are formed.
-                const float x_max = e0f * invz, s_max = z_others * invz;
+                // are what this code adds (q^l = (1 + beta) w / (z + beta w), w = the other codes' sum); the units are put
+                // back when the totals are formed.
 #pragma unroll
                 for (int j = 0; j < JV; ++j) {
                     const int vi = tid + j * NT;
@@ -360,19 +370,20 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                         Elem<T>::load(reinterpret_cast<const T *>(rstage + (size_t)vi * 16), rho);
 #pragma unroll
                         for (int q = 0; q < VEC; ++q) {
-                            const CodeRadius kr = code_radius_fast<RAW>(rho[q], a.r_max, beta_max);
-                            if (e[j * VEC + q] == e0f) {
-                                const float den_l = fmaf(kr.alpha, s_max, kr.a), den_u = fmaf(kr.beta, x_max, 1.0f);
-                                const float rden = rcp_approx(den_l * den_u);
-                                const float ql = s_max * den_u * rden, d = kr.bma * (x_max * s_max * rden);
+                            const float ev = e[j * VEC + q];
+                            const float beta = code_beta<RAW>(rho[q], a.r_max, beta_max);
+                            float pl, d;
+                            if (ev == e0f) {
+                                code_bounds(ev, z_others, zf, beta, pl, d);  // w = z - e from the other codes' sum
+                                const float den_l = fmaf(beta, z_others, zf);
+                                const float ql = (z_others + beta * z_others) * rcp_approx(den_l);
                                 sA += d;
                                 sB -= ql;
                                 sAA = fmaf(d, d, sAA);
                                 sAB = fmaf(d, 1.0f - ql, sAB);
                                 sBB += fmaf(ql, ql, -2.0f * ql);
                             } else {
-                                float pl, d;
-                                code_bounds(e[j * VEC + q] * invz, kr, pl, d);
+                                code_bounds(ev, zf - ev, zf, beta, pl, d);
                                 sA += d;
                                 sB += pl;
                                 sAA = fmaf(d, d, sAA);
@@ -427,7 +438,8 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
 #pragma unroll
                     for (int q = 0; q < VEC; ++q) {
                         float pl, d;
-                        code_bounds(e[j * VEC + q] * invz, code_radius_fast<RAW>(rho[q], a.r_max, beta_max), pl, d);
+                        const float ev = e[j * VEC + q];
+                        code_bounds(ev, zf - ev, zf, code_beta<RAW>(rho[q], a.r_max, beta_max), pl, d);
                         const float x = fmaf(fku, d, fg * pl) - fmu;
                         sd = fmaf(x, x, sd);
                     }
@@ -503,6 +515,7 @@ bool quantify_percode_eligible(const QuantifyArgs &a, int dtype)
     if (a.rm.pos != nullptr) return false;  // decode row maps stay on the general kernel
     if (a.out.dense_p || a.out.dense_lo || a.out.dense_up) return false;
     if (a.vb % vec != 0 || a.n % vec != 0) return false;
+    if (a.r_max > 30.0f) return false;  // the product of the two denominators must stay in float range: beta <= e^30
     return a.n >= 2048 && (a.n / vec) * 16 <= kPcRowBytes;
 }
 
