@@ -2,14 +2,16 @@
 // a row's logits AND its radii arrive together through a ring of shared-memory stages filled by bulk (TMA) copies,
 // so both tensors are read from HBM exactly once.
 //
-// One persistent CTA of 32 warps per SM walks rows blockIdx.x, blockIdx.x + gridDim.x, ...; thread 0 issues the two
-// copies of a row three rows ahead.  A landed row is swept three times from shared memory: the maximum; one
-// exponential per code (kept in registers, 16 per thread) with the softmax and entropy sums; then both InterFuse
-// bounds of every code from its own radius, with the five sums Omega and Sigma are built from.  Each sweep ends in
-// a CTA barrier that publishes the per-warp sums; every thread then holds the row's totals.  A row whose widths are
-// nearly uniform gets a fourth sweep that sums (delta - mu)^2 directly (the moment form would cancel).  The row's
-// totals are parked in shared memory; every 32 rows each warp finishes one parked row (logarithm, square root,
-// flag, stores), so that no single thread's scalar work holds up the CTA row after row.
+// One persistent CTA per SM walks rows blockIdx.x, blockIdx.x + gridDim.x, ...  Its 32 warps form two groups of 16
+// that take these rows in turn, each group with its own named barrier and scratch, so that while one group stands
+// at a barrier or in a reduction the other keeps the pipes busy.  A group sweeps its landed row three times from
+// shared memory: the maximum; one exponential per code with the softmax and entropy sums; then both InterFuse
+// bounds of every code from its own radius (the exponential formed again: nothing per code is kept in registers),
+// with the five sums Omega and Sigma are built from.  Each sweep ends in a group barrier that publishes the
+// per-warp sums; every thread of the group then holds the row's totals in float.  A row whose widths are nearly
+// uniform gets a fourth sweep that sums (delta - mu)^2 directly (the moment form would cancel).  The row's totals
+// are parked in shared memory; every 16 rows each warp of the group finishes one parked row in double (logarithm,
+// square root, flag, stores).  The thread that ends a row's last sweep issues the copies of the row three further on.
 #include "quantify_finish.cuh"
 
 namespace ciar {
@@ -17,18 +19,20 @@ namespace ciar {
 namespace {
 
 constexpr int kPcThreads = 1024;
-constexpr int kPcWarps = kPcThreads / 32;
+constexpr int kPcGroups = 2;
+constexpr int kPcGT = kPcThreads / kPcGroups;  // threads of a group
+constexpr int kPcGW = kPcGT / 32;              // warps of a group; as many rows are parked before they are finished
 constexpr int kPcStages = 3;
-constexpr int kPcJV = 2;          // 16-byte vectors of a row per thread, at most
+constexpr int kPcJV = 4;            // 16-byte vectors of a row per thread, at most
 constexpr int kPcRowBytes = 32768;  // widest row of one tensor a stage takes (16384 bf16 / 8192 fp32 codes)
-constexpr int kBarPc = 1;
+constexpr int kBarPc = 1;           // named barriers kBarPc + group
 
 // A row's totals in double: the softmax sums as computed (relative to m2 = fl(m * log2e)) and the five interval sums.
 struct PcTotals {
     double z_raw, t_raw, A, B, AA, AB, BB;
 };
 
-// A row whose sweeps are done: what the finishing arithmetic needs.
+// A row whose sweeps are done: what the finishing arithmetic needs (a dominant code's unit is already in the totals).
 struct PcParked {
     PcTotals tt;
     double dev;  // sum of (delta - mu)^2 from the fourth sweep, when low_cv
@@ -36,35 +40,56 @@ struct PcParked {
     float m;
     int first, low_cv;
 };
-// (the totals of a parked row already hold a dominant code's unit)
+
+// Scratch of one group.
+struct PcGroup {
+    PcParked park[kPcGW];
+    float wmax[kPcGW];
+    float zs[kPcGW], ts[kPcGW];  // per-warp sums of the sweeps
+    float sums[5][kPcGW];
+    float dev[kPcGW];
+    int cnt, first;  // codes counted as the row maximum, and the lowest code equal to it
+    int abort;       // a wait of this group ran out (set before the group's barrier, read after it: uniform)
+};
 
 struct PcShared {
     unsigned long long full[kPcStages];
-    PcParked park[kPcWarps];
-    float wmax[kPcWarps];
-    float zs[kPcWarps], ts[kPcWarps];  // per-warp sums of the sweeps
-    float sums[5][kPcWarps];
-    float dev[kPcWarps];
-    int cnt, first;  // codes equal to the row maximum, and the lowest of them
-    int abort;
+    PcGroup grp[kPcGroups];
 };
 
+// Sum over the 16 per-warp values of a group (every lane gets it).
+__device__ __forceinline__ float group_sum_f(const float *v, int lane)
+{
+    float x = v[lane & (kPcGW - 1)];
+#pragma unroll
+    for (int o = kPcGW / 2; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+__device__ __forceinline__ double group_sum_d(const float *v, int lane)
+{
+    double x = (double)v[lane & (kPcGW - 1)];
+#pragma unroll
+    for (int o = kPcGW / 2; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
 // The per-warp sums of a row joined in double (a warp; every lane gets the totals).  The exponent actually used is
-// c * log2e_f - m2 = (c - m) * log2e_f + off with off = m * log2e_f - m2; a code equal to the maximum, left out of
+// c * log2e_f - m2 = (c - m) * log2e_f + off with off = m * log2e_f - m2; a code counted as the maximum, left out of
 // the sweeps' sums, contributes exactly 2^off to z_raw and 2^off off to t_raw.  A dominant code (see the kernel) entered
 // the sums of p^l and p^l^2 less 1.
-__device__ __forceinline__ PcTotals row_totals(const PcShared &sh, int lane, float m, int nmax, int dominant)
+__device__ __forceinline__ PcTotals row_totals(const PcGroup &gs, int lane, float m, int nmax, int dominant)
 {
     const double off = (double)m * (double)kLog2e - (double)(m * kLog2e);
     const double scale = exp2(off);
     PcTotals t;
-    t.z_raw = warp_sum_d((double)sh.zs[lane]) + (double)nmax * scale;
-    t.t_raw = warp_sum_d((double)sh.ts[lane]) + (double)nmax * scale * off;
-    t.A = warp_sum_d((double)sh.sums[0][lane]);
-    t.B = warp_sum_d((double)sh.sums[1][lane]) + (double)dominant;
-    t.AA = warp_sum_d((double)sh.sums[2][lane]);
-    t.AB = warp_sum_d((double)sh.sums[3][lane]);
-    t.BB = warp_sum_d((double)sh.sums[4][lane]) + (double)dominant;
+    t.z_raw = group_sum_d(gs.zs, lane) + (double)nmax * scale;
+    t.t_raw = group_sum_d(gs.ts, lane) + (double)nmax * scale * off;
+    t.A = group_sum_d(gs.sums[0], lane);
+    t.B = group_sum_d(gs.sums[1], lane) + (double)dominant;
+    t.AA = group_sum_d(gs.sums[2], lane);
+    t.AB = group_sum_d(gs.sums[3], lane);
+    t.BB = group_sum_d(gs.sums[4], lane) + (double)dominant;
     return t;
 }
 
@@ -128,29 +153,33 @@ __device__ __forceinline__ void code_bounds(float e, float w, float z, float bet
 template <typename T, bool RAW>
 __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const __grid_constant__ QuantifyArgs a)
 {
-    constexpr int NT = kPcThreads, NW = kPcWarps, JV = kPcJV;
-    static_assert(NW == 32, "a lane reads one warp's share");
+    constexpr int GT = kPcGT, GW = kPcGW, JV = kPcJV;
     constexpr int VEC = Elem<T>::kVec;
     extern __shared__ __align__(128) unsigned char smem[];
     const int nvec = a.n / VEC;
     const uint32_t row_bytes = (uint32_t)nvec * 16u;
     const size_t stage_bytes = 2 * (size_t)row_bytes;  // logits, then radii
     PcShared &sh = *reinterpret_cast<PcShared *>(smem + kPcStages * stage_bytes);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int grp = threadIdx.x / GT, gtid = threadIdx.x % GT, lane = gtid & 31, gwarp = gtid >> 5;
+    const int bar = kBarPc + grp;
+    PcGroup &gs = sh.grp[grp];
     const ciar_quantify_out &o = a.out;
 
-    if (tid == 0) {
+    if (threadIdx.x == 0) {
 #pragma unroll
         for (int s = 0; s < kPcStages; ++s) mbar_init(&sh.full[s], 1);
-        sh.abort = 0;
-        sh.cnt = 0;
-        sh.first = INT_MAX;
         mbar_init_fence();
+    }
+    if (gtid == 0) {
+        gs.abort = 0;
+        gs.cnt = 0;
+        gs.first = INT_MAX;
     }
     __syncthreads();
 
+    // The CTA's k-th row; the groups take k = 0, 1, 2, ... in turn, row k lands in stage k % kPcStages.
     auto row_of = [&](int k) -> int64_t { return blockIdx.x + (int64_t)k * gridDim.x; };
-    auto issue = [&](int k) {  // thread 0 only
+    auto issue = [&](int k) {  // one thread
         const int64_t lr = row_of(k);
         if (lr < a.rows) {
             const int s = k % kPcStages;
@@ -161,17 +190,17 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
             bulk_copy_g2s(stage + row_bytes, reinterpret_cast<const T *>(a.radius) + at, row_bytes, &sh.full[s]);
         }
     };
-    if (tid == 0) {
+    if (threadIdx.x == 0) {
 #pragma unroll
         for (int s = 0; s < kPcStages; ++s) issue(s);
     }
 
     const double nn = (double)a.n;
-    // Lane 0 of every warp finishes one parked row.
+    // Lane 0 of every warp of the group finishes one parked row.
     auto finish_parked = [&](int count) {
-        named_bar_sync(kBarPc, NT);
-        if (warp < count && lane == 0) {
-            const PcParked &p = sh.park[warp];
+        named_bar_sync(bar, GT);
+        if (gwarp < count && lane == 0) {
+            const PcParked &p = gs.park[gwarp];
             const PcTotals &tt = p.tt;
             const PcScales sc = row_scales(tt, a.lo_cap, a.hi_cap, nn);
             double var = (sc.k_up * sc.k_up * tt.AA + 2.0 * sc.k_up * sc.g * tt.AB + sc.g * sc.g * tt.BB) / nn - sc.mu * sc.mu;
@@ -212,48 +241,46 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
     };
 
     const float beta_max = (float)expm1((double)a.r_max);
-    int filled = 0;
     const float inv_n = 1.0f / (float)a.n;
-    uint32_t phases = 0;
+    int filled = 0;
     bool aborted = false;
-    int k = 0;
-    for (; row_of(k) < a.rows; ++k) {
+    int k = grp;
+    for (; row_of(k) < a.rows; k += kPcGroups) {
         const int s = k % kPcStages;
         const unsigned char *stage = smem + s * stage_bytes;
         const unsigned char *rstage = stage + row_bytes;
-        if (mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kWaitCycles)) phases ^= 1u << s;
-        else sh.abort = 1;
+        // the stage's phases complete in the order of its rows k, k + 3, k + 6, ...: this row's has parity (k / 3) & 1
+        if (!mbar_wait_bounded(&sh.full[s], (uint32_t)(k / kPcStages) & 1u, kWaitCycles)) gs.abort = 1;
 
         // ---- sweep 1: the maximum
         {
             typename Vec<T>::Max mx = Vec<T>::max_init();
 #pragma unroll
             for (int j = 0; j < JV; ++j) {
-                const int vi = tid + j * NT;
+                const int vi = gtid + j * GT;
                 if (vi < nvec) mx = Vec<T>::fold_max(mx, stage_vec(stage, vi));
             }
             const float wm = warp_redux_max(Vec<T>::max_value(mx));
-            if (lane == 0) sh.wmax[warp] = wm;
+            if (lane == 0) gs.wmax[gwarp] = wm;
         }
-        named_bar_sync(kBarPc, NT);
-        if (sh.abort) {
+        named_bar_sync(bar, GT);
+        if (gs.abort) {
             aborted = true;
             break;
         }
-        const float m = warp_redux_max(sh.wmax[lane]);
+        const float m = warp_redux_max(gs.wmax[lane & (GW - 1)]);
         const float m2 = m * kLog2e;
 
-        // ---- sweep 2: exponentials (kept), their sum and the entropy sum.  Codes whose exponential equals the
+        // ---- sweep 2: the sum of the exponentials and the entropy sum.  Codes whose exponential equals the
         // maximum's are counted: their terms, 2^off each, enter exactly when the totals are formed.
         const float e0f = ex2_approx(fmaf(m, kLog2e, -m2));
-        float e[JV * VEC];
         bool has_max;  // this thread holds a code counted as a maximum
         {
             float z = 0.f, t = 0.f;
             int cnt = 0;
 #pragma unroll
             for (int j = 0; j < JV; ++j) {
-                const int vi = tid + j * NT;
+                const int vi = gtid + j * GT;
                 if (vi < nvec) {
                     float c[VEC];
                     Elem<T>::load(reinterpret_cast<const T *>(stage + (size_t)vi * 16), c);
@@ -261,7 +288,6 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                     for (int q = 0; q < VEC; ++q) {
                         const float d = fmaf(c[q], kLog2e, -m2);
                         const float ev = ex2_approx(d);  // a NaN logit poisons z on purpose
-                        e[j * VEC + q] = ev;
                         if (ev == e0f) {
                             ++cnt;
                         } else {
@@ -269,9 +295,6 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                             t = fmaf(ev, d, t);  // 0 * -inf = NaN for a -inf logit: redone below
                         }
                     }
-                } else {
-#pragma unroll
-                    for (int q = 0; q < VEC; ++q) e[j * VEC + q] = 0.f;
                 }
             }
             has_max = cnt > 0;
@@ -281,7 +304,7 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                 // -inf logit (exponential 0, exponent -inf) or a real NaN forms it again with such products taken
                 // as 0 (a real NaN still shows in the sum of exponentials).
                 t = 0.f;
-                for (int vi = tid; vi < nvec; vi += NT) {
+                for (int vi = gtid; vi < nvec; vi += GT) {
                     const T *cp = reinterpret_cast<const T *>(stage + (size_t)vi * 16);
 #pragma unroll 1
                     for (int q = 0; q < VEC; ++q) {
@@ -293,26 +316,25 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                 }
             }
             const float zt = warp_sum_pair(z, t, lane);  // lanes 0..15: z, lanes 16..31: t
-            if (lane == 0) sh.zs[warp] = zt;
-            if (lane == 16) sh.ts[warp] = zt;
-            if (__any_sync(0xffffffffu, cnt > 0)) {
+            if (lane == 0) gs.zs[gwarp] = zt;
+            if (lane == 16) gs.ts[gwarp] = zt;
+            if (__any_sync(0xffffffffu, has_max)) {
 #pragma unroll
                 for (int ofs = 16; ofs > 0; ofs >>= 1) {
                     cnt += __shfl_xor_sync(0xffffffffu, cnt, ofs);
                     first = min(first, __shfl_xor_sync(0xffffffffu, first, ofs));
                 }
                 if (lane == 0) {
-                    atomicAdd(&sh.cnt, cnt);
-                    atomicMin(&sh.first, first);
+                    atomicAdd(&gs.cnt, cnt);
+                    atomicMin(&gs.first, first);
                 }
             }
         }
-        named_bar_sync(kBarPc, NT);
-        // Every thread needs the row's sum only in float (for 1 / z); the totals in double are formed once, by
-        // warp 0, when it parks the row.  off = m * log2e - m2 is the rounding error of m2; a code equal to the
-        // maximum contributes 2^off.
-        const int nmax = sh.cnt, first = sh.first;
-        const float z_others = warp_sum_f(sh.zs[lane]);
+        named_bar_sync(bar, GT);
+        // Every thread needs the row's sum only in float; the totals in double are formed once, by the group's
+        // first warp, when it parks the row.
+        const int nmax = gs.cnt, first = gs.first;
+        const float z_others = group_sum_f(gs.zs, lane);
         const float zf = z_others + (float)nmax * e0f;
 
         int status = 0;
@@ -320,34 +342,35 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         else if (!(zf < INFINITY) || !(zf > 0.f)) status |= CIAR_ROW_NAN;  // NaN or +inf logit
         if (status) {
             // nothing more is read from the stage: hand it to the row three further on
-            named_bar_sync(kBarPc, NT);
-            if (tid == 0) {
+            named_bar_sync(bar, GT);
+            if (gtid == 0) {
                 write_unusable(o, row_of(k), status);
-                sh.cnt = 0;
-                sh.first = INT_MAX;
+                gs.cnt = 0;
+                gs.first = INT_MAX;
                 fence_proxy_async_smem();
                 issue(k + kPcStages);
             }
             continue;
         }
-
-        // ---- sweep 3: both bounds of every code from its own radius; the sums of d, p^l, d^2, d p^l, p^l^2
         // A single code that holds more than half of the mass: its p^l, near 1, would cost the sum of the lower bounds
         // (which decides Omega = 1.01 - S_lo when S_lo < 0.99) its last digits in float.
         const int dominant = nmax == 1 && e0f > 0.5f * zf;
+
+        // ---- sweep 3: both bounds of every code from its own radius; the sums of d, p^l, d^2, d p^l, p^l^2
         {
             float sA = 0.f, sB = 0.f, sAA = 0.f, sAB = 0.f, sBB = 0.f;
             if (!(dominant && has_max)) {
 #pragma unroll
                 for (int j = 0; j < JV; ++j) {
-                    const int vi = tid + j * NT;
+                    const int vi = gtid + j * GT;
                     if (vi < nvec) {
-                        float rho[VEC];
+                        float c[VEC], rho[VEC];
+                        Elem<T>::load(reinterpret_cast<const T *>(stage + (size_t)vi * 16), c);
                         Elem<T>::load(reinterpret_cast<const T *>(rstage + (size_t)vi * 16), rho);
 #pragma unroll
                         for (int q = 0; q < VEC; ++q) {
                             float pl, d;
-                            const float ev = e[j * VEC + q];
+                            const float ev = ex2_approx(fmaf(c[q], kLog2e, -m2));
                             code_bounds(ev, zf - ev, zf, code_beta<RAW>(rho[q], a.r_max, beta_max), pl, d);
                             sA += d;
                             sB += pl;
@@ -358,61 +381,55 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                     }
                 }
             } else {
-                // The one thread that holds the dominant code.  With s = 1 - x taken from the other codes' sum,
-                // 1 - p^l = s / (a + alpha s) =: q^l keeps its digits, so p^l - 1 = -q^l and p^l^2 - 1 = q^l^2 - 2 q^l
-                // are what this code adds (q^l = (1 + beta) w / (z + beta w), w = the other codes' sum); the units are put
-                // back when the totals are formed.
-#pragma unroll
-                for (int j = 0; j < JV; ++j) {
-                    const int vi = tid + j * NT;
-                    if (vi < nvec) {
-                        float rho[VEC];
-                        Elem<T>::load(reinterpret_cast<const T *>(rstage + (size_t)vi * 16), rho);
-#pragma unroll
-                        for (int q = 0; q < VEC; ++q) {
-                            const float ev = e[j * VEC + q];
-                            const float beta = code_beta<RAW>(rho[q], a.r_max, beta_max);
-                            float pl, d;
-                            if (ev == e0f) {
-                                code_bounds(ev, z_others, zf, beta, pl, d);  // w = z - e from the other codes' sum
-                                const float den_l = fmaf(beta, z_others, zf);
-                                const float ql = (z_others + beta * z_others) * rcp_approx(den_l);
-                                sA += d;
-                                sB -= ql;
-                                sAA = fmaf(d, d, sAA);
-                                sAB = fmaf(d, 1.0f - ql, sAB);
-                                sBB += fmaf(ql, ql, -2.0f * ql);
-                            } else {
-                                code_bounds(ev, zf - ev, zf, beta, pl, d);
-                                sA += d;
-                                sB += pl;
-                                sAA = fmaf(d, d, sAA);
-                                sAB = fmaf(d, pl, sAB);
-                                sBB = fmaf(pl, pl, sBB);
-                            }
+                // The one thread that holds the dominant code.  With w = z - e taken from the other codes' sum,
+                // 1 - p^l = (1 + beta) w / (z + beta w) =: q^l keeps its digits, so p^l - 1 = -q^l and
+                // p^l^2 - 1 = q^l^2 - 2 q^l are what this code adds; the units are put back when the totals are formed.
+                for (int vi = gtid; vi < nvec; vi += GT) {
+                    const T *cp = reinterpret_cast<const T *>(stage + (size_t)vi * 16);
+                    const T *rp = reinterpret_cast<const T *>(rstage + (size_t)vi * 16);
+#pragma unroll 1
+                    for (int q = 0; q < VEC; ++q) {
+                        const float ev = ex2_approx(fmaf(Elem<T>::widen(cp[q]), kLog2e, -m2));
+                        const float beta = code_beta<RAW>(Elem<T>::widen(rp[q]), a.r_max, beta_max);
+                        float pl, d;
+                        if (ev == e0f) {
+                            code_bounds(ev, z_others, zf, beta, pl, d);
+                            const float ql = (z_others + beta * z_others) * rcp_approx(fmaf(beta, z_others, zf));
+                            sA += d;
+                            sB -= ql;
+                            sAA = fmaf(d, d, sAA);
+                            sAB = fmaf(d, 1.0f - ql, sAB);
+                            sBB += fmaf(ql, ql, -2.0f * ql);
+                        } else {
+                            code_bounds(ev, zf - ev, zf, beta, pl, d);
+                            sA += d;
+                            sB += pl;
+                            sAA = fmaf(d, d, sAA);
+                            sAB = fmaf(d, pl, sAB);
+                            sBB = fmaf(pl, pl, sBB);
                         }
                     }
                 }
             }
             const float r0 = warp_sum_pair(sA, sB, lane), r1 = warp_sum_pair(sAA, sAB, lane), r2 = warp_sum_f(sBB);
             if (lane == 0) {
-                sh.sums[0][warp] = r0;
-                sh.sums[2][warp] = r1;
-                sh.sums[4][warp] = r2;
+                gs.sums[0][gwarp] = r0;
+                gs.sums[2][gwarp] = r1;
+                gs.sums[4][gwarp] = r2;
             }
             if (lane == 16) {
-                sh.sums[1][warp] = r0;
-                sh.sums[3][warp] = r1;
+                gs.sums[1][gwarp] = r0;
+                gs.sums[3][gwarp] = r1;
             }
         }
-        named_bar_sync(kBarPc, NT);
+        named_bar_sync(bar, GT);
         // A look at the totals in float, only to see whether the moment form of the variance is safe for this row
         // (every thread forms the same values, so the branch below is uniform).
         bool low_cv;
         {
-            const float A = warp_sum_f(sh.sums[0][lane]), B = warp_sum_f(sh.sums[1][lane]) + (float)dominant,
-                        AA = warp_sum_f(sh.sums[2][lane]), AB = warp_sum_f(sh.sums[3][lane]),
-                        BB = warp_sum_f(sh.sums[4][lane]) + (float)dominant;
+            const float A = group_sum_f(gs.sums[0], lane), B = group_sum_f(gs.sums[1], lane) + (float)dominant,
+                        AA = group_sum_f(gs.sums[2], lane), AB = group_sum_f(gs.sums[3], lane),
+                        BB = group_sum_f(gs.sums[4], lane) + (float)dominant;
             const float S_lo = B, S_up = A + B;
             float k_lo = 1.f, k_up = 1.f;
             if (S_lo > 0.f && a.lo_cap < S_lo) k_lo = a.lo_cap * rcp_approx(S_lo);
@@ -425,20 +442,21 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         double dev_total = 0.0;
         if (low_cv) {
             // ---- sweep 4 (rare): sum of (delta_i - mu)^2 with the scales known, from the totals in double
-            const PcTotals tt = row_totals(sh, lane, m, nmax, dominant);
+            const PcTotals tt = row_totals(gs, lane, m, nmax, dominant);
             const PcScales sc = row_scales(tt, a.lo_cap, a.hi_cap, nn);
             const float fku = (float)sc.k_up, fg = (float)sc.g, fmu = (float)sc.mu;
             float sd = 0.f;
 #pragma unroll
             for (int j = 0; j < JV; ++j) {
-                const int vi = tid + j * NT;
+                const int vi = gtid + j * GT;
                 if (vi < nvec) {
-                    float rho[VEC];
+                    float c[VEC], rho[VEC];
+                    Elem<T>::load(reinterpret_cast<const T *>(stage + (size_t)vi * 16), c);
                     Elem<T>::load(reinterpret_cast<const T *>(rstage + (size_t)vi * 16), rho);
 #pragma unroll
                     for (int q = 0; q < VEC; ++q) {
                         float pl, d;
-                        const float ev = e[j * VEC + q];
+                        const float ev = ex2_approx(fmaf(c[q], kLog2e, -m2));
                         code_bounds(ev, zf - ev, zf, code_beta<RAW>(rho[q], a.r_max, beta_max), pl, d);
                         const float x = fmaf(fku, d, fg * pl) - fmu;
                         sd = fmaf(x, x, sd);
@@ -446,20 +464,20 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                 }
             }
             sd = warp_sum_f(sd);
-            if (lane == 0) sh.dev[warp] = sd;
-            named_bar_sync(kBarPc, NT);
-            if (warp == 0) dev_total = warp_sum_d((double)sh.dev[lane]);
+            if (lane == 0) gs.dev[gwarp] = sd;
+            named_bar_sync(bar, GT);
+            if (gwarp == 0) dev_total = group_sum_d(gs.dev, lane);
         }
-        if (tid == 0) {  // every thread has read the stage for the last time: refill it
-            sh.cnt = 0;
-            sh.first = INT_MAX;
+        if (gtid == 0) {  // every thread of the group has read the stage for the last time: refill it
+            gs.cnt = 0;
+            gs.first = INT_MAX;
             fence_proxy_async_smem();
             issue(k + kPcStages);
         }
-        if (warp == 0) {  // park the row's totals
-            const PcTotals tt = row_totals(sh, lane, m, nmax, dominant);
+        if (gwarp == 0) {  // park the row's totals
+            const PcTotals tt = row_totals(gs, lane, m, nmax, dominant);
             if (lane == 0) {
-                PcParked &p = sh.park[filled];
+                PcParked &p = gs.park[filled];
                 p.tt = tt;
                 p.dev = dev_total;
                 p.lr = row_of(k);
@@ -468,18 +486,25 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                 p.low_cv = low_cv;
             }
         }
-        if (++filled == NW) {
+        if (++filled == GW) {
             finish_parked(filled);
             filled = 0;
         }
     }
     if (filled > 0) finish_parked(filled);
 
-    if (aborted && tid == 0) {
-        // A copy never arrived.  Mark this row and the rest of this CTA's rows, then give the copies still in
-        // flight a last bounded chance to land before the CTA leaves.
-        for (int k2 = k; row_of(k2) < a.rows; ++k2) write_unusable(o, row_of(k2), CIAR_ROW_TIMEOUT);
-        for (int s = 0; s < kPcStages; ++s) mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kDrainCycles);
+    if (aborted && gtid == 0) {
+        // A copy never arrived: mark this row and the rest of this group's rows.
+        for (int k2 = k; row_of(k2) < a.rows; k2 += kPcGroups) write_unusable(o, row_of(k2), CIAR_ROW_TIMEOUT);
+    }
+    __syncthreads();
+    if ((sh.grp[0].abort | sh.grp[1].abort) && threadIdx.x == 0) {
+        // Give the copies still in flight a last bounded chance to land before the CTA leaves (of the two waits on
+        // a stage, the one for a phase already complete returns at once).
+        for (int s = 0; s < kPcStages; ++s) {
+            mbar_wait_bounded(&sh.full[s], 0u, kDrainCycles);
+            mbar_wait_bounded(&sh.full[s], 1u, kDrainCycles);
+        }
     }
 }
 
