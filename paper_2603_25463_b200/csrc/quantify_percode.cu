@@ -138,6 +138,18 @@ __device__ __forceinline__ float code_beta(float rho, float r_max, float beta_ma
     return expm1_fast(!(rho > r_max) ? rho : r_max);
 }
 
+// code_beta for two codes: the scaling of the exponent is packed, the rest is per code
+template <bool RAW>
+__device__ __forceinline__ float2 code_beta2(float2 rho, float r_max, float beta_max)
+{
+    if (RAW) {
+        const float2 x = __fmul2_rn(rho, make_float2(kLog2e, kLog2e));
+        const float ux = ex2_approx(x.x), uy = ex2_approx(x.y);
+        return make_float2(!(ux > beta_max) ? ux : beta_max, !(uy > beta_max) ? uy : beta_max);
+    }
+    return make_float2(code_beta<false>(rho.x, r_max, beta_max), code_beta<false>(rho.y, r_max, beta_max));
+}
+
 // One code's raw bounds from its exponential e (any common scale), the row's sum z of them and w = z - e:
 //   p^l = e / (z + beta w),   p^u = (1 + beta) e / (z + beta e),
 //   d = p^u - p^l = beta (2 + beta) e w / ((z + beta w)(z + beta e))   -- no cancellation for small radii.
@@ -155,6 +167,7 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
 {
     constexpr int GT = kPcGT, GW = kPcGW, JV = kPcJV;
     constexpr int VEC = Elem<T>::kVec;
+    constexpr int NPV = Vec<T>::kPairs;  // float2 pairs per 16-byte vector
     extern __shared__ __align__(128) unsigned char smem[];
     const int nvec = a.n / VEC;
     const uint32_t row_bytes = (uint32_t)nvec * 16u;
@@ -276,27 +289,33 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         const float e0f = ex2_approx(fmaf(m, kLog2e, -m2));
         bool has_max;  // this thread holds a code counted as a maximum
         {
-            float z = 0.f, t = 0.f;
+            float2 z2 = f2(0.f), t2 = f2(0.f);
             int cnt = 0;
+            const float2 L2 = f2(kLog2e), nm2 = f2(-m2);
 #pragma unroll
             for (int j = 0; j < JV; ++j) {
                 const int vi = gtid + j * GT;
                 if (vi < nvec) {
-                    float c[VEC];
-                    Elem<T>::load(reinterpret_cast<const T *>(stage + (size_t)vi * 16), c);
+                    float2 c[NPV];
+                    Vec<T>::pairs(stage_vec(stage, vi), c);
 #pragma unroll
-                    for (int q = 0; q < VEC; ++q) {
-                        const float d = fmaf(c[q], kLog2e, -m2);
-                        const float ev = ex2_approx(d);  // a NaN logit poisons z on purpose
-                        if (ev == e0f) {
+                    for (int q = 0; q < NPV; ++q) {
+                        const float2 d = __ffma2_rn(c[q], L2, nm2);
+                        float2 ev = make_float2(ex2_approx(d.x), ex2_approx(d.y));  // a NaN logit poisons z on purpose
+                        if (ev.x == e0f) {
                             ++cnt;
-                        } else {
-                            z += ev;
-                            t = fmaf(ev, d, t);  // 0 * -inf = NaN for a -inf logit: redone below
+                            ev.x = 0.f;
                         }
+                        if (ev.y == e0f) {
+                            ++cnt;
+                            ev.y = 0.f;
+                        }
+                        z2 = __fadd2_rn(z2, ev);
+                        t2 = __ffma2_rn(ev, d, t2);  // 0 * -inf = NaN for a -inf logit: redone below
                     }
                 }
             }
+            float z = z2.x + z2.y, t = t2.x + t2.y;
             has_max = cnt > 0;
             int first = INT_MAX;
             if (has_max || !(t == t)) {
@@ -360,26 +379,41 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         {
             float sA = 0.f, sB = 0.f, sAA = 0.f, sAB = 0.f, sBB = 0.f;
             if (!(dominant && has_max)) {
+                // two codes at a time in packed fp32 (the exponentials, reciprocals and clamps stay scalar)
+                float2 pA = f2(0.f), pB = f2(0.f), pAA = f2(0.f), pAB = f2(0.f), pBB = f2(0.f);
+                const float2 L2 = f2(kLog2e), nm2 = f2(-m2), zf2 = f2(zf), neg1 = f2(-1.0f);
 #pragma unroll
                 for (int j = 0; j < JV; ++j) {
                     const int vi = gtid + j * GT;
                     if (vi < nvec) {
-                        float c[VEC], rho[VEC];
-                        Elem<T>::load(reinterpret_cast<const T *>(stage + (size_t)vi * 16), c);
-                        Elem<T>::load(reinterpret_cast<const T *>(rstage + (size_t)vi * 16), rho);
+                        float2 c[NPV], rho[NPV];
+                        Vec<T>::pairs(stage_vec(stage, vi), c);
+                        Vec<T>::pairs(stage_vec(rstage, vi), rho);
 #pragma unroll
-                        for (int q = 0; q < VEC; ++q) {
-                            float pl, d;
-                            const float ev = ex2_approx(fmaf(c[q], kLog2e, -m2));
-                            code_bounds(ev, zf - ev, zf, code_beta<RAW>(rho[q], a.r_max, beta_max), pl, d);
-                            sA += d;
-                            sB += pl;
-                            sAA = fmaf(d, d, sAA);
-                            sAB = fmaf(d, pl, sAB);
-                            sBB = fmaf(pl, pl, sBB);
+                        for (int q = 0; q < NPV; ++q) {
+                            const float2 x = __ffma2_rn(c[q], L2, nm2);
+                            const float2 ev = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                            const float2 beta = code_beta2<RAW>(rho[q], a.r_max, beta_max);
+                            const float2 w = __ffma2_rn(ev, neg1, zf2);
+                            const float2 den_l = __ffma2_rn(beta, w, zf2), den_u = __ffma2_rn(beta, ev, zf2);
+                            const float2 pr = __fmul2_rn(den_l, den_u);
+                            const float2 rd = make_float2(rcp_approx(pr.x), rcp_approx(pr.y));
+                            const float2 pl = __fmul2_rn(ev, __fmul2_rn(rd, den_u));
+                            const float2 kd = __ffma2_rn(beta, beta, __fadd2_rn(beta, beta));
+                            const float2 d = __fmul2_rn(__fmul2_rn(kd, rd), __fmul2_rn(ev, w));
+                            pA = __fadd2_rn(pA, d);
+                            pB = __fadd2_rn(pB, pl);
+                            pAA = __ffma2_rn(d, d, pAA);
+                            pAB = __ffma2_rn(d, pl, pAB);
+                            pBB = __ffma2_rn(pl, pl, pBB);
                         }
                     }
                 }
+                sA = pA.x + pA.y;
+                sB = pB.x + pB.y;
+                sAA = pAA.x + pAA.y;
+                sAB = pAB.x + pAB.y;
+                sBB = pBB.x + pBB.y;
             } else {
                 // The one thread that holds the dominant code.  With w = z - e taken from the other codes' sum,
                 // 1 - p^l = (1 + beta) w / (z + beta w) =: q^l keeps its digits, so p^l - 1 = -q^l and
