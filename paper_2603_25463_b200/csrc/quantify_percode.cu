@@ -12,6 +12,8 @@
 // uniform gets a fourth sweep that sums (delta - mu)^2 directly (the moment form would cancel).  The row's totals
 // are parked in shared memory; every 16 rows each warp of the group finishes one parked row in double (logarithm,
 // square root, flag, stores).  The thread that ends a row's last sweep issues the copies of the row three further on.
+#include <type_traits>
+
 #include "quantify_finish.cuh"
 
 namespace ciar {
@@ -318,18 +320,28 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
             float z = z2.x + z2.y, t = t2.x + t2.y;
             has_max = cnt > 0;
             int first = INT_MAX;
-            if (has_max || !(t == t)) {
-                // A thread that holds a maximum looks for the lowest code equal to it; one whose entropy sum met a
-                // -inf logit (exponential 0, exponent -inf) or a real NaN forms it again with such products taken
-                // as 0 (a real NaN still shows in the sum of exponentials).
+            if (has_max) {  // the lowest code of this thread equal to the maximum
+#pragma unroll
+                for (int j = 0; j < JV; ++j) {
+                    const int vi = gtid + j * GT;
+                    if (vi < nvec) {
+                        float c[VEC];
+                        Elem<T>::load(reinterpret_cast<const T *>(stage + (size_t)vi * 16), c);
+#pragma unroll
+                        for (int q = VEC - 1; q >= 0; --q)
+                            if (c[q] == m) first = min(first, vi * VEC + q);
+                    }
+                }
+            }
+            if (!(t == t)) {
+                // The entropy sum met a -inf logit (exponential 0, exponent -inf) or a real NaN: it is formed again with
+                // such products taken as 0 (a real NaN still shows in the sum of exponentials).
                 t = 0.f;
                 for (int vi = gtid; vi < nvec; vi += GT) {
                     const T *cp = reinterpret_cast<const T *>(stage + (size_t)vi * 16);
 #pragma unroll 1
                     for (int q = 0; q < VEC; ++q) {
-                        const float c = Elem<T>::widen(cp[q]);
-                        const float d = fmaf(c, kLog2e, -m2), ev = ex2_approx(d);
-                        if (c == m) first = min(first, vi * VEC + q);
+                        const float d = fmaf(Elem<T>::widen(cp[q]), kLog2e, -m2), ev = ex2_approx(d);
                         if (ev != e0f) t = fmaf(ev, fmaxf(d, kNegHuge), t);
                     }
                 }
@@ -377,10 +389,12 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
 
         // ---- sweep 3: both bounds of every code from its own radius; the sums of d, p^l, d^2, d p^l, p^l^2
         {
-            float sA = 0.f, sB = 0.f, sAA = 0.f, sAB = 0.f, sBB = 0.f;
-            if (!(dominant && has_max)) {
-                // two codes at a time in packed fp32 (the exponentials, reciprocals and clamps stay scalar)
-                float2 pA = f2(0.f), pB = f2(0.f), pAA = f2(0.f), pAB = f2(0.f), pBB = f2(0.f);
+            // two codes at a time in packed fp32 (the exponentials, reciprocals and clamps stay scalar)
+            float2 pA = f2(0.f), pB = f2(0.f), pAA = f2(0.f), pAB = f2(0.f), pBB = f2(0.f);
+            float dom_rho = 0.f;
+            bool dom_here = false;  // this thread holds the dominant code
+            auto sweep = [&](auto look_out) {
+                constexpr bool DOM = decltype(look_out)::value;
                 const float2 L2 = f2(kLog2e), nm2 = f2(-m2), zf2 = f2(zf), neg1 = f2(-1.0f);
 #pragma unroll
                 for (int j = 0; j < JV; ++j) {
@@ -392,7 +406,19 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
 #pragma unroll
                         for (int q = 0; q < NPV; ++q) {
                             const float2 x = __ffma2_rn(c[q], L2, nm2);
-                            const float2 ev = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                            float2 ev = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                            if (DOM) {  // the dominant code is taken out here (its terms become 0) and put in below
+                                if (ev.x == e0f) {
+                                    dom_rho = rho[q].x;
+                                    dom_here = true;
+                                    ev.x = 0.f;
+                                }
+                                if (ev.y == e0f) {
+                                    dom_rho = rho[q].y;
+                                    dom_here = true;
+                                    ev.y = 0.f;
+                                }
+                            }
                             const float2 beta = code_beta2<RAW>(rho[q], a.r_max, beta_max);
                             const float2 w = __ffma2_rn(ev, neg1, zf2);
                             const float2 den_l = __ffma2_rn(beta, w, zf2), den_u = __ffma2_rn(beta, ev, zf2);
@@ -409,41 +435,24 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                         }
                     }
                 }
-                sA = pA.x + pA.y;
-                sB = pB.x + pB.y;
-                sAA = pAA.x + pAA.y;
-                sAB = pAB.x + pAB.y;
-                sBB = pBB.x + pBB.y;
-            } else {
-                // The one thread that holds the dominant code.  With w = z - e taken from the other codes' sum,
-                // 1 - p^l = (1 + beta) w / (z + beta w) =: q^l keeps its digits, so p^l - 1 = -q^l and
-                // p^l^2 - 1 = q^l^2 - 2 q^l are what this code adds; the units are put back when the totals are formed.
-                for (int vi = gtid; vi < nvec; vi += GT) {
-                    const T *cp = reinterpret_cast<const T *>(stage + (size_t)vi * 16);
-                    const T *rp = reinterpret_cast<const T *>(rstage + (size_t)vi * 16);
-#pragma unroll 1
-                    for (int q = 0; q < VEC; ++q) {
-                        const float ev = ex2_approx(fmaf(Elem<T>::widen(cp[q]), kLog2e, -m2));
-                        const float beta = code_beta<RAW>(Elem<T>::widen(rp[q]), a.r_max, beta_max);
-                        float pl, d;
-                        if (ev == e0f) {
-                            code_bounds(ev, z_others, zf, beta, pl, d);
-                            const float ql = (z_others + beta * z_others) * rcp_approx(fmaf(beta, z_others, zf));
-                            sA += d;
-                            sB -= ql;
-                            sAA = fmaf(d, d, sAA);
-                            sAB = fmaf(d, 1.0f - ql, sAB);
-                            sBB += fmaf(ql, ql, -2.0f * ql);
-                        } else {
-                            code_bounds(ev, zf - ev, zf, beta, pl, d);
-                            sA += d;
-                            sB += pl;
-                            sAA = fmaf(d, d, sAA);
-                            sAB = fmaf(d, pl, sAB);
-                            sBB = fmaf(pl, pl, sBB);
-                        }
-                    }
-                }
+            };
+            // only the warp that holds a dominant code pays for looking out for it (the branch is uniform in a warp)
+            if (dominant && __any_sync(0xffffffffu, has_max)) sweep(std::true_type());
+            else sweep(std::false_type());
+            float sA = pA.x + pA.y, sB = pB.x + pB.y, sAA = pAA.x + pAA.y, sAB = pAB.x + pAB.y, sBB = pBB.x + pBB.y;
+            if (dom_here) {
+                // With w = z - e taken from the other codes' sum, 1 - p^l = (1 + beta) w / (z + beta w) =: q^l keeps its
+                // digits, so p^l - 1 = -q^l and p^l^2 - 1 = q^l^2 - 2 q^l are what the dominant code adds; the units are
+                // put back when the totals are formed.
+                const float beta = code_beta<RAW>(dom_rho, a.r_max, beta_max);
+                float pl, d;
+                code_bounds(e0f, z_others, zf, beta, pl, d);
+                const float ql = (z_others + beta * z_others) * rcp_approx(fmaf(beta, z_others, zf));
+                sA += d;
+                sB -= ql;
+                sAA = fmaf(d, d, sAA);
+                sAB = fmaf(d, 1.0f - ql, sAB);
+                sBB += fmaf(ql, ql, -2.0f * ql);
             }
             const float r0 = warp_sum_pair(sA, sB, lane), r1 = warp_sum_pair(sAA, sAB, lane), r2 = warp_sum_f(sBB);
             if (lane == 0) {
