@@ -34,22 +34,21 @@ struct PcTotals {
     double z_raw, t_raw, A, B, AA, AB, BB;
 };
 
-// A row whose sweeps are done: what the finishing arithmetic needs (a dominant code's unit is already in the totals).
+// A row whose sweeps are done: the per-warp sums as the sweeps left them (joined in double when the row is finished)
+// and the row's scalars.
 struct PcParked {
-    PcTotals tt;
-    double dev;  // sum of (delta - mu)^2 from the fourth sweep, when low_cv
+    float zs[kPcGW], ts[kPcGW];  // sum of exponentials (maximum codes left out), entropy sum
+    float sums[5][kPcGW];        // d, p^l, d^2, d p^l, p^l^2 (a dominant code's p^l terms less 1)
+    float dev[kPcGW];            // sum of (delta - mu)^2 from the fourth sweep, when low_cv
     long long lr;
     float m;
-    int first, low_cv;
+    int first, nmax, dominant, low_cv;
 };
 
 // Scratch of one group.
 struct PcGroup {
     PcParked park[kPcGW];
     float wmax[kPcGW];
-    float zs[kPcGW], ts[kPcGW];  // per-warp sums of the sweeps
-    float sums[5][kPcGW];
-    float dev[kPcGW];
     int cnt, first;  // codes counted as the row maximum, and the lowest code equal to it
     int abort;       // a wait of this group ran out (set before the group's barrier, read after it: uniform)
 };
@@ -80,7 +79,7 @@ __device__ __forceinline__ double group_sum_d(const float *v, int lane)
 // c * log2e_f - m2 = (c - m) * log2e_f + off with off = m * log2e_f - m2; a code counted as the maximum, left out of
 // the sweeps' sums, contributes exactly 2^off to z_raw and 2^off off to t_raw.  A dominant code (see the kernel) entered
 // the sums of p^l and p^l^2 less 1.
-__device__ __forceinline__ PcTotals row_totals(const PcGroup &gs, int lane, float m, int nmax, int dominant)
+__device__ __forceinline__ PcTotals row_totals(const PcParked &gs, int lane, float m, int nmax, int dominant)
 {
     const double off = (double)m * (double)kLog2e - (double)(m * kLog2e);
     const double scale = exp2(off);
@@ -211,15 +210,17 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
     }
 
     const double nn = (double)a.n;
-    // Lane 0 of every warp of the group finishes one parked row.
+    // Every warp of the group finishes one parked row: it joins the per-warp sums in double, lane 0 does the rest.
     auto finish_parked = [&](int count) {
         named_bar_sync(bar, GT);
-        if (gwarp < count && lane == 0) {
+        if (gwarp < count) {
             const PcParked &p = gs.park[gwarp];
-            const PcTotals &tt = p.tt;
+            const PcTotals tt = row_totals(p, lane, p.m, p.nmax, p.dominant);
+            const double dev = group_sum_d(p.dev, lane);
+            if (lane != 0) return;
             const PcScales sc = row_scales(tt, a.lo_cap, a.hi_cap, nn);
             double var = (sc.k_up * sc.k_up * tt.AA + 2.0 * sc.k_up * sc.g * tt.AB + sc.g * sc.g * tt.BB) / nn - sc.mu * sc.mu;
-            if (p.low_cv) var = p.dev / nn;
+            if (p.low_cv) var = dev / nn;
             const float m = p.m;
             const double off = (double)m * (double)kLog2e - (double)(m * kLog2e);
             const double unscale = exp2(-off);
@@ -264,6 +265,7 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         const int s = k % kPcStages;
         const unsigned char *stage = smem + s * stage_bytes;
         const unsigned char *rstage = stage + row_bytes;
+        PcParked &pk = gs.park[filled];  // the sweeps leave their per-warp sums in the row's parking slot
         // the stage's phases complete in the order of its rows k, k + 3, k + 6, ...: this row's has parity (k / 3) & 1
         if (!mbar_wait_bounded(&sh.full[s], (uint32_t)(k / kPcStages) & 1u, kWaitCycles)) gs.abort = 1;
 
@@ -347,8 +349,8 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                 }
             }
             const float zt = warp_sum_pair(z, t, lane);  // lanes 0..15: z, lanes 16..31: t
-            if (lane == 0) gs.zs[gwarp] = zt;
-            if (lane == 16) gs.ts[gwarp] = zt;
+            if (lane == 0) pk.zs[gwarp] = zt;
+            if (lane == 16) pk.ts[gwarp] = zt;
             if (__any_sync(0xffffffffu, has_max)) {
 #pragma unroll
                 for (int ofs = 16; ofs > 0; ofs >>= 1) {
@@ -362,10 +364,9 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
             }
         }
         named_bar_sync(bar, GT);
-        // Every thread needs the row's sum only in float; the totals in double are formed once, by the group's
-        // first warp, when it parks the row.
+        // Every thread needs the row's sum only in float; the totals in double are formed when the row is finished.
         const int nmax = gs.cnt, first = gs.first;
-        const float z_others = group_sum_f(gs.zs, lane);
+        const float z_others = group_sum_f(pk.zs, lane);
         const float zf = z_others + (float)nmax * e0f;
 
         int status = 0;
@@ -456,13 +457,13 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
             }
             const float r0 = warp_sum_pair(sA, sB, lane), r1 = warp_sum_pair(sAA, sAB, lane), r2 = warp_sum_f(sBB);
             if (lane == 0) {
-                gs.sums[0][gwarp] = r0;
-                gs.sums[2][gwarp] = r1;
-                gs.sums[4][gwarp] = r2;
+                pk.sums[0][gwarp] = r0;
+                pk.sums[2][gwarp] = r1;
+                pk.sums[4][gwarp] = r2;
             }
             if (lane == 16) {
-                gs.sums[1][gwarp] = r0;
-                gs.sums[3][gwarp] = r1;
+                pk.sums[1][gwarp] = r0;
+                pk.sums[3][gwarp] = r1;
             }
         }
         named_bar_sync(bar, GT);
@@ -470,9 +471,9 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         // (every thread forms the same values, so the branch below is uniform).
         bool low_cv;
         {
-            const float A = group_sum_f(gs.sums[0], lane), B = group_sum_f(gs.sums[1], lane) + (float)dominant,
-                        AA = group_sum_f(gs.sums[2], lane), AB = group_sum_f(gs.sums[3], lane),
-                        BB = group_sum_f(gs.sums[4], lane) + (float)dominant;
+            const float A = group_sum_f(pk.sums[0], lane), B = group_sum_f(pk.sums[1], lane) + (float)dominant,
+                        AA = group_sum_f(pk.sums[2], lane), AB = group_sum_f(pk.sums[3], lane),
+                        BB = group_sum_f(pk.sums[4], lane) + (float)dominant;
             const float S_lo = B, S_up = A + B;
             float k_lo = 1.f, k_up = 1.f;
             if (S_lo > 0.f && a.lo_cap < S_lo) k_lo = a.lo_cap * rcp_approx(S_lo);
@@ -482,10 +483,9 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
             const float var = (k_up * k_up * AA + 2.f * k_up * g * AB + g * g * BB) * inv_n - mu * mu;
             low_cv = !(var >= 0.1f * mu * mu);  // nearly uniform widths: the moment form cancels
         }
-        double dev_total = 0.0;
         if (low_cv) {
             // ---- sweep 4 (rare): sum of (delta_i - mu)^2 with the scales known, from the totals in double
-            const PcTotals tt = row_totals(gs, lane, m, nmax, dominant);
+            const PcTotals tt = row_totals(pk, lane, m, nmax, dominant);
             const PcScales sc = row_scales(tt, a.lo_cap, a.hi_cap, nn);
             const float fku = (float)sc.k_up, fg = (float)sc.g, fmu = (float)sc.mu;
             float sd = 0.f;
@@ -507,27 +507,20 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                 }
             }
             sd = warp_sum_f(sd);
-            if (lane == 0) gs.dev[gwarp] = sd;
+            if (lane == 0) pk.dev[gwarp] = sd;
             named_bar_sync(bar, GT);
-            if (gwarp == 0) dev_total = group_sum_d(gs.dev, lane);
         }
-        if (gtid == 0) {  // every thread of the group has read the stage for the last time: refill it
+        if (gtid == 0) {  // every thread of the group has read the stage for the last time: refill it; the row's scalars
             gs.cnt = 0;
             gs.first = INT_MAX;
             fence_proxy_async_smem();
             issue(k + kPcStages);
-        }
-        if (gwarp == 0) {  // park the row's totals
-            const PcTotals tt = row_totals(gs, lane, m, nmax, dominant);
-            if (lane == 0) {
-                PcParked &p = gs.park[filled];
-                p.tt = tt;
-                p.dev = dev_total;
-                p.lr = row_of(k);
-                p.m = m;
-                p.first = first;
-                p.low_cv = low_cv;
-            }
+            pk.lr = row_of(k);
+            pk.m = m;
+            pk.first = first;
+            pk.nmax = nmax;
+            pk.dominant = dominant;
+            pk.low_cv = low_cv;
         }
         if (++filled == GW) {
             finish_parked(filled);
