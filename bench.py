@@ -254,7 +254,7 @@ def run_ours(args):
     v_name = "verify_plan+accept_wide+window" if wide else "verify_plan+accept+window"
     dominant = q_name if q_ms >= v_ms else v_name
     dom_gbs = q_gbs if q_ms >= v_ms else v_gbs
-    traffic = None if per_code else load_traffic(dominant, args.workload)
+    traffic = None if args.images else load_traffic(dominant, args.workload)  # the captures are of full batches
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
                 "frac": dom_gbs / peak, "peak_kind": "of " + peak_kind, "traffic": traffic,
                 "frac_of_nominal_8TBs": dom_gbs / NOMINAL_HBM_GBS,
@@ -284,6 +284,8 @@ def run_ours(args):
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/, keyed by (kernel, workload).  An entry is dropped (-> null) when its kernel changes after the capture.
 NCU_TRAFFIC = {
+    # captured on 2304 of the 9216 rows and scaled by the rows: profiles/quantify_percode_kernel_llamagen384.md
+    ("quantify_percode_kernel", "llamagen384"): 4 * (151.1e6 + 4.0e6),
     ("quantify_stream_kernel", "llamagen384"): 303.5e6 + 8.4e6,  # profiles/quantify_stream_kernel_llamagen384.md
     # captured on 2048 of the 65536 rows and scaled by the rows (every row is handled alone): profiles/quantify_wide_kernel_largevocab.md
     ("quantify_wide_kernel", "largevocab"): 32 * (1078.2e6 + 12.5e6),
