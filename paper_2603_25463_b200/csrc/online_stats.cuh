@@ -101,8 +101,7 @@ __device__ __forceinline__ void online_sweep(OnlineStats &st, const unsigned cha
                     if (ev == e0w) ++cnt; else zz += ev;
                 }
                 zz = warp_sum_f(zz);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+                cnt = __reduce_add_sync(0xffffffffu, cnt);
                 if (lane == h) {
                     zs = zz;
                     st.cnt += cnt;

@@ -352,11 +352,8 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
             if (lane == 0) pk.zs[gwarp] = zt;
             if (lane == 16) pk.ts[gwarp] = zt;
             if (__any_sync(0xffffffffu, has_max)) {
-#pragma unroll
-                for (int ofs = 16; ofs > 0; ofs >>= 1) {
-                    cnt += __shfl_xor_sync(0xffffffffu, cnt, ofs);
-                    first = min(first, __shfl_xor_sync(0xffffffffu, first, ofs));
-                }
+                cnt = __reduce_add_sync(0xffffffffu, cnt);
+                first = __reduce_min_sync(0xffffffffu, first);
                 if (lane == 0) {
                     atomicAdd(&gs.cnt, cnt);
                     atomicMin(&gs.first, first);

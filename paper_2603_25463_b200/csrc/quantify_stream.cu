@@ -236,11 +236,8 @@ __global__ void __launch_bounds__(NT, MINB) quantify_stream_kernel(const __grid_
                     if (c == m) first = min(first, vi * VEC + i % VEC);
                 }
                 zz = warp_sum_f(zz);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-                    first = min(first, __shfl_xor_sync(0xffffffffu, first, o));
-                }
+                cnt = __reduce_add_sync(0xffffffffu, cnt);
+                first = __reduce_min_sync(0xffffffffu, first);
                 if (lane == h) zs = zz;
                 if (lane == 0) {
                     if (cnt > 0) atomicAdd(&sh.nmax[it & 3], cnt);

@@ -304,8 +304,7 @@ __global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __gri
                 if (ev == e0) ++cnt; else zz += ev;
             }
             zz = warp_sum_f(zz);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+            cnt = __reduce_add_sync(0xffffffffu, cnt);
             if (lane == h) zs = zz;
             if (lane == 0 && cnt > 0) atomicAdd(&sh.nmax[k & 3], cnt);
         }
