@@ -7,8 +7,8 @@
 // at a barrier or in a reduction the other keeps the pipes busy.  A group sweeps its landed row three times from
 // shared memory: the maximum; one exponential per code with the softmax and entropy sums; then both InterFuse
 // bounds of every code from its own radius (the exponential formed again: nothing per code is kept in registers),
-// with the five sums Omega and Sigma are built from.  Each sweep ends in a group barrier that publishes the
-// per-warp sums; every thread of the group then holds the row's totals in float.  A row whose widths are nearly
+// with the five sums Omega and Sigma are built from.  The second and third sweep end in a group barrier that publishes
+// the per-warp sums (the first sweep of a row runs before the last barrier of the group's row before it); every thread of the group then holds the row's totals in float.  A row whose widths are nearly
 // uniform gets a fourth sweep that sums (delta - mu)^2 directly (the moment form would cancel).  The row's totals
 // are parked in shared memory; every 16 rows each warp of the group finishes one parked row in double (logarithm,
 // square root, flag, stores).  The thread that ends a row's last sweep issues the copies of the row three further on.
@@ -48,7 +48,7 @@ struct PcParked {
 // Scratch of one group.
 struct PcGroup {
     PcParked park[kPcGW];
-    float wmax[kPcGW];
+    float wmax[2][kPcGW];  // by the row's turn: a row's maxima are written while the row before it is still in use
     int cnt, first;  // codes counted as the row maximum, and the lowest code equal to it
     int abort;       // a wait of this group ran out (set before the group's barrier, read after it: uniform)
 };
@@ -261,31 +261,36 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
     int filled = 0;
     bool aborted = false;
     int k = grp;
-    for (; row_of(k) < a.rows; k += kPcGroups) {
+    // Waits for the CTA's kk-th row to land and takes the maximum over it (sweep 1); each warp's maximum goes to the
+    // given slot.  It runs one row ahead, before the last barrier of the group's row before, so that barrier also
+    // publishes these maxima.  (The stage's phases complete in the order of its rows kk, kk + 3, kk + 6, ...: this
+    // row's has parity (kk / 3) & 1.)
+    auto first_sweep = [&](int kk, int slot) {
+        const int s = kk % kPcStages;
+        const unsigned char *stage = smem + s * stage_bytes;
+        if (!mbar_wait_bounded(&sh.full[s], (uint32_t)(kk / kPcStages) & 1u, kWaitCycles)) gs.abort = 1;
+        typename Vec<T>::Max mx = Vec<T>::max_init();
+#pragma unroll
+        for (int j = 0; j < JV; ++j) {
+            const int vi = gtid + j * GT;
+            if (vi < nvec) mx = Vec<T>::fold_max(mx, stage_vec(stage, vi));
+        }
+        const float wm = warp_redux_max(Vec<T>::max_value(mx));
+        if (lane == 0) gs.wmax[slot][gwarp] = wm;
+    };
+    int it = 0;  // rows this group has started: its low bit picks the slot of the per-warp maxima
+    if (row_of(k) < a.rows) {
+        first_sweep(k, 0);
+        named_bar_sync(bar, GT);
+        if (gs.abort) aborted = true;
+    }
+    for (; row_of(k) < a.rows && !aborted; k += kPcGroups, ++it) {
         const int s = k % kPcStages;
         const unsigned char *stage = smem + s * stage_bytes;
         const unsigned char *rstage = stage + row_bytes;
         PcParked &pk = gs.park[filled];  // the sweeps leave their per-warp sums in the row's parking slot
-        // the stage's phases complete in the order of its rows k, k + 3, k + 6, ...: this row's has parity (k / 3) & 1
-        if (!mbar_wait_bounded(&sh.full[s], (uint32_t)(k / kPcStages) & 1u, kWaitCycles)) gs.abort = 1;
-
-        // ---- sweep 1: the maximum
-        {
-            typename Vec<T>::Max mx = Vec<T>::max_init();
-#pragma unroll
-            for (int j = 0; j < JV; ++j) {
-                const int vi = gtid + j * GT;
-                if (vi < nvec) mx = Vec<T>::fold_max(mx, stage_vec(stage, vi));
-            }
-            const float wm = warp_redux_max(Vec<T>::max_value(mx));
-            if (lane == 0) gs.wmax[gwarp] = wm;
-        }
-        named_bar_sync(bar, GT);
-        if (gs.abort) {
-            aborted = true;
-            break;
-        }
-        const float m = warp_redux_max(gs.wmax[lane & (GW - 1)]);
+        const bool more = row_of(k + kPcGroups) < a.rows;  // the group has a row after this one
+        const float m = warp_redux_max(gs.wmax[it & 1][lane & (GW - 1)]);
         const float m2 = m * kLog2e;
 
         // ---- sweep 2: the sum of the exponentials and the entropy sum.  Codes whose exponential equals the
@@ -371,6 +376,7 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         else if (!(zf < INFINITY) || !(zf > 0.f)) status |= CIAR_ROW_NAN;  // NaN or +inf logit
         if (status) {
             // nothing more is read from the stage: hand it to the row three further on
+            if (more) first_sweep(k + kPcGroups, (it + 1) & 1);
             named_bar_sync(bar, GT);
             if (gtid == 0) {
                 write_unusable(o, row_of(k), status);
@@ -378,6 +384,11 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                 gs.first = INT_MAX;
                 fence_proxy_async_smem();
                 issue(k + kPcStages);
+            }
+            if (more && gs.abort) {  // the next row never landed
+                aborted = true;
+                k += kPcGroups;
+                break;
             }
             continue;
         }
@@ -463,7 +474,9 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
                 pk.sums[3][gwarp] = r1;
             }
         }
+        if (more) first_sweep(k + kPcGroups, (it + 1) & 1);  // sweep 1 of the group's next row
         named_bar_sync(bar, GT);
+        const bool next_abort = more && gs.abort;  // set only by this group's threads, before the barrier: uniform
         // A look at the totals in float, only to see whether the moment form of the variance is safe for this row
         // (every thread forms the same values, so the branch below is uniform).
         bool low_cv;
@@ -522,6 +535,11 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         if (++filled == GW) {
             finish_parked(filled);
             filled = 0;
+        }
+        if (next_abort) {  // the next row never landed
+            aborted = true;
+            k += kPcGroups;
+            break;
         }
     }
     if (filled > 0) finish_parked(filled);
