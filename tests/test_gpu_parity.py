@@ -468,10 +468,15 @@ def test_workload_largevocab_sample(ciar):
 
 # ---------------------------------------------------------------- decode loop
 
-def _decode_compare(ciar, wl, mode=oracle.VERIFY_ANCHORED, pos0=0, max_steps=None, stop_at_near_tie=False):
-    inp = synth.make_inputs(wl)
+def _decode_compare(ciar, wl, mode=oracle.VERIFY_ANCHORED, pos0=0, max_steps=None, stop_at_near_tie=False,
+                    per_code=False):
+    inp = synth.make_inputs(wl, per_code_radius=per_code)
     seq, req = wl.tokens_per_image, wl.images
-    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
+    if per_code:
+        prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_CODE, radius=inp.radius_code, radius_is_raw=True,
+                                    tau=wl.tau)
+    else:
+        prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
     ost = oracle.DecodeState(req, seq, pos0)
     gst = ciar.DecodeState.allocate(req, seq, "cuda")
     ciar.decode_init(gst, pos0)
@@ -523,6 +528,13 @@ def test_decode_loop_many_requests_finishing_at_different_steps(ciar):
     wl = synth.Workload("dec3", 168, 4, 5, 2048, "bf16", 8, 0.5, seed=15, decode=True, tau=1e-3)  # 1344 rows per step, 20 tokens
     steps, ost = _decode_compare(ciar, wl)
     assert steps >= 3 and (ost.pos == wl.tokens_per_image).all()
+
+
+def test_decode_loop_per_code_radius(ciar):
+    """The decode loop with a pool of raw per-code radii indexed like the logit pools."""
+    wl = synth.Workload("dec6", 12, 4, 6, 2048, "bf16", 8, 0.5, seed=17, decode=True, tau=1e-3)  # 24 tokens
+    steps, ost = _decode_compare(ciar, wl, per_code=True, stop_at_near_tie=True)
+    assert steps >= 1
 
 
 def test_decode_loop_wide_rows(ciar):
