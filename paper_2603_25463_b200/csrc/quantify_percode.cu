@@ -7,11 +7,13 @@
 // at a barrier or in a reduction the other keeps the pipes busy.  A group sweeps its landed row three times from
 // shared memory: the maximum; one exponential per code with the softmax and entropy sums; then both InterFuse
 // bounds of every code from its own radius (the exponential formed again: nothing per code is kept in registers),
-// with the five sums Omega and Sigma are built from.  The second and third sweep end in a group barrier that publishes
-// the per-warp sums (the first sweep of a row runs before the last barrier of the group's row before it); every thread of the group then holds the row's totals in float.  A row whose widths are nearly
-// uniform gets a fourth sweep that sums (delta - mu)^2 directly (the moment form would cancel).  The row's totals
-// are parked in shared memory; every 16 rows each warp of the group finishes one parked row in double (logarithm,
-// square root, flag, stores).  The thread that ends a row's last sweep issues the copies of the row three further on.
+// with the five sums Omega and Sigma are built from.  The second and third sweep end in a group barrier that
+// publishes the per-warp sums (the first sweep of a row runs before the last barrier of the group's row before it);
+// every thread of the group then holds the row's totals in float.  A row whose widths are nearly uniform gets a
+// fourth sweep that sums (delta - mu)^2 directly (the moment form would cancel).  The sweeps leave their per-warp
+// sums in the row's parking slot; every 16 rows each warp of the group joins one parked row's sums in double and
+// finishes it (logarithm, square root, flag, stores).  The thread that ends a row's last sweep issues the copies of
+// the row three further on.
 #include <type_traits>
 
 #include "quantify_finish.cuh"
