@@ -30,6 +30,7 @@ constexpr int kPcStages = 3;
 constexpr int kPcJV = 4;            // 16-byte vectors of a row per thread, at most
 constexpr int kPcRowBytes = 32768;  // widest row of one tensor a stage takes (16384 bf16 / 8192 fp32 codes)
 constexpr int kBarPc = 1;           // named barriers kBarPc + group
+constexpr int kPcListCap = 1024;    // rows a CTA may walk when the rows go through a position map (decode mode)
 
 // A row's totals in double: the softmax sums as computed (relative to m2 = fl(m * log2e)) and the five interval sums.
 struct PcTotals {
@@ -58,6 +59,9 @@ struct PcGroup {
 struct PcShared {
     unsigned long long full[kPcStages];
     PcGroup grp[kPcGroups];
+    // decode mode: which of this CTA's rows (as multiples of the grid) hold something to quantify
+    int nlist;
+    int list[kPcListCap];
 };
 
 // Sum over the 16 per-warp values of a group (every lane gets it).
@@ -184,6 +188,7 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
     if (threadIdx.x == 0) {
 #pragma unroll
         for (int s = 0; s < kPcStages; ++s) mbar_init(&sh.full[s], 1);
+        sh.nlist = 0;
         mbar_init_fence();
     }
     if (gtid == 0) {
@@ -192,15 +197,43 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
         gs.first = INT_MAX;
     }
     __syncthreads();
+    // Decode mode: the rows go through a position map, and a position past the end of its sequence holds nothing to
+    // quantify.  Such rows get their outputs here; the others are listed (in any order: rows are independent), and
+    // the CTA walks the list.
+    const bool mapped = a.rm.pos != nullptr;
+    if (mapped) {
+        const int nk = (int)((a.rows - blockIdx.x + gridDim.x - 1) / gridDim.x);  // at most kPcListCap (checked by the host)
+        for (int i = threadIdx.x; i < nk; i += kPcThreads) {
+            const int64_t lr = blockIdx.x + (int64_t)i * gridDim.x;
+            int64_t pr;
+            if (map_row(a.rm, lr, pr)) {
+                sh.list[atomicAdd(&sh.nlist, 1)] = i;
+            } else {
+                if (o.flag) o.flag[lr] = 0;
+                if (o.row_status) o.row_status[lr] = 0;
+            }
+        }
+        __syncthreads();
+    }
+    const int nlist = mapped ? sh.nlist : 0;
 
-    // The CTA's k-th row; the groups take k = 0, 1, 2, ... in turn, row k lands in stage k % kPcStages.
-    auto row_of = [&](int k) -> int64_t { return blockIdx.x + (int64_t)k * gridDim.x; };
+    // The CTA's k-th row (a.rows when it has no more); the groups take k = 0, 1, 2, ... in turn, row k lands in
+    // stage k % kPcStages.
+    auto row_of = [&](int k) -> int64_t {
+        if (mapped) return k < nlist ? blockIdx.x + (int64_t)sh.list[k] * gridDim.x : a.rows;
+        return blockIdx.x + (int64_t)k * gridDim.x;
+    };
+    auto phys_row = [&](int64_t lr) -> int64_t {
+        int64_t pr = lr;
+        if (mapped) map_row(a.rm, lr, pr);
+        return pr;
+    };
     auto issue = [&](int k) {  // one thread
         const int64_t lr = row_of(k);
         if (lr < a.rows) {
             const int s = k % kPcStages;
             unsigned char *stage = smem + s * stage_bytes;
-            const size_t at = (size_t)(a.vb + lr * a.row_stride);
+            const size_t at = (size_t)(a.vb + phys_row(lr) * a.row_stride);
             mbar_arrive_expect_tx(&sh.full[s], 2 * row_bytes);
             bulk_copy_g2s(stage, reinterpret_cast<const T *>(a.logits) + at, row_bytes, &sh.full[s]);
             bulk_copy_g2s(stage + row_bytes, reinterpret_cast<const T *>(a.radius) + at, row_bytes, &sh.full[s]);
@@ -239,7 +272,7 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
             case CIAR_POLICY_INTERVAL: fl = score > (double)a.tau; break;
             case CIAR_POLICY_ENTROPY: fl = entropy > (double)a.tau; break;
             case CIAR_POLICY_MAXPROB: fl = p_max < (double)a.tau; break;
-            case CIAR_POLICY_RANDOM: fl = a.u_flag[lr] < a.tau; break;
+            case CIAR_POLICY_RANDOM: fl = a.u_flag[phys_row(lr)] < a.tau; break;
             default: fl = 1; break;
             }
             if (o.row_max) o.row_max[lr] = m;
@@ -590,7 +623,10 @@ bool quantify_percode_eligible(const QuantifyArgs &a, int dtype)
 {
     const int vec = dtype == CIAR_F32 ? 4 : 8;
     if (a.radius_mode != CIAR_RADIUS_PER_CODE) return false;
-    if (a.rm.pos != nullptr) return false;  // decode row maps stay on the general kernel
+    if (a.rm.pos != nullptr) {  // decode row map: a CTA lists its rows, and the list is of fixed size
+        const int64_t grid = a.rows < sm_count() ? a.rows : sm_count();
+        if (grid > 0 && (a.rows + grid - 1) / grid > kPcListCap) return false;
+    }
     if (a.out.dense_p || a.out.dense_lo || a.out.dense_up) return false;
     if (a.vb % vec != 0 || a.n % vec != 0) return false;
     if (a.r_max > 30.0f) return false;  // the product of the two denominators must stay in float range: beta <= e^30
