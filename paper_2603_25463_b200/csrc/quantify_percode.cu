@@ -169,7 +169,8 @@ __device__ __forceinline__ void code_bounds(float e, float w, float z, float bet
     d = (fmaf(beta, beta, beta + beta) * rd) * (e * w);
 }
 
-template <typename T, bool RAW>
+// MAPPED: the rows go through a position map (decode mode).
+template <typename T, bool RAW, bool MAPPED>
 __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const __grid_constant__ QuantifyArgs a)
 {
     constexpr int GT = kPcGT, GW = kPcGW, JV = kPcJV;
@@ -200,7 +201,7 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
     // Decode mode: the rows go through a position map, and a position past the end of its sequence holds nothing to
     // quantify.  Such rows get their outputs here; the others are listed (in any order: rows are independent), and
     // the CTA walks the list.
-    const bool mapped = a.rm.pos != nullptr;
+    constexpr bool mapped = MAPPED;
     if (mapped) {
         const int nk = (int)((a.rows - blockIdx.x + gridDim.x - 1) / gridDim.x);  // at most kPcListCap (checked by the host)
         for (int i = threadIdx.x; i < nk; i += kPcThreads) {
@@ -594,7 +595,7 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
     }
 }
 
-template <typename T, bool RAW>
+template <typename T, bool RAW, bool MAPPED>
 cudaError_t launch_pc(const QuantifyArgs &a, cudaStream_t stream)
 {
     constexpr size_t smem_max = (size_t)kPcStages * 2 * kPcRowBytes + sizeof(PcShared);
@@ -604,7 +605,7 @@ cudaError_t launch_pc(const QuantifyArgs &a, cudaStream_t stream)
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        err = cudaFuncSetAttribute(quantify_percode_kernel<T, RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+        err = cudaFuncSetAttribute(quantify_percode_kernel<T, RAW, MAPPED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
         if (err != cudaSuccess) return err;
         configured[dev] = true;
     }
@@ -612,7 +613,7 @@ cudaError_t launch_pc(const QuantifyArgs &a, cudaStream_t stream)
     const size_t smem = (size_t)kPcStages * 2 * row_bytes + sizeof(PcShared);
     const int64_t cap = sm_count();
     const unsigned grid = (unsigned)(a.rows < cap ? a.rows : cap);
-    quantify_percode_kernel<T, RAW><<<grid, kPcThreads, smem, stream>>>(a);
+    quantify_percode_kernel<T, RAW, MAPPED><<<grid, kPcThreads, smem, stream>>>(a);
     count_launch();
     return cudaGetLastError();
 }
@@ -636,9 +637,13 @@ bool quantify_percode_eligible(const QuantifyArgs &a, int dtype)
 cudaError_t launch_quantify_percode(const QuantifyArgs &a, int dtype, cudaStream_t stream)
 {
     if (a.rows == 0) return cudaSuccess;
-    if (dtype == CIAR_F32)
-        return a.radius_is_raw ? launch_pc<float, true>(a, stream) : launch_pc<float, false>(a, stream);
-    return a.radius_is_raw ? launch_pc<__nv_bfloat16, true>(a, stream) : launch_pc<__nv_bfloat16, false>(a, stream);
+    const bool raw = a.radius_is_raw != 0, mapped = a.rm.pos != nullptr;
+    if (dtype == CIAR_F32) {
+        if (mapped) return raw ? launch_pc<float, true, true>(a, stream) : launch_pc<float, false, true>(a, stream);
+        return raw ? launch_pc<float, true, false>(a, stream) : launch_pc<float, false, false>(a, stream);
+    }
+    if (mapped) return raw ? launch_pc<__nv_bfloat16, true, true>(a, stream) : launch_pc<__nv_bfloat16, false, true>(a, stream);
+    return raw ? launch_pc<__nv_bfloat16, true, false>(a, stream) : launch_pc<__nv_bfloat16, false, false>(a, stream);
 }
 
 }  // namespace ciar
