@@ -323,9 +323,13 @@ def run_decode(args):
     wl = ciar_dist.rank_workload(synth.WORKLOADS["decode"], rank)
     if args.decode_requests:
         wl = wl.scaled(images=args.decode_requests)
-    inp = synth.make_inputs(wl, device=dev)
+    per_code = args.radius == "per_code"
+    inp = synth.make_inputs(wl, device=dev, per_code_radius=per_code)
     req, seq = wl.images, wl.tokens_per_image
-    params = ciar.IntervalParams(radius_mode=ciar.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
+    if per_code:  # a pool of raw per-code radii indexed like the logit pools
+        params = ciar.IntervalParams(radius_mode=ciar.RADIUS_PER_CODE, radius=inp.radius_code, radius_is_raw=True, tau=wl.tau)
+    else:
+        params = ciar.IntervalParams(radius_mode=ciar.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
     state = ciar.DecodeState.allocate(req, seq, dev)
     ws = ciar.alloc_workspace(req * wl.window, wl.window, dev)
 
@@ -402,7 +406,7 @@ def run_decode(args):
         "config": {"workload": "decode", "requests_per_gpu": req, "seq_len": seq, "vocab": wl.vocab, "logits": wl.dtype,
                    "window": wl.window, "verify_mode": "anchored", "radius": args.radius, "tau": wl.tau,
                    "launch": "cuda graph replay" if graph is not None else "direct",
-                   "l2": "pools of %.1f GB, rows touched once" % (2 * req * seq * wl.vocab * wl.elem_bytes / 1e9)},
+                   "l2": "pools of %.1f GB, rows touched once" % ((3 if per_code else 2) * req * seq * wl.vocab * wl.elem_bytes / 1e9)},
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
         "gpu_launches": int(launches),
