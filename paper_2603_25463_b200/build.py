@@ -1,20 +1,26 @@
-"""Builds ``libciar.so`` (the C-ABI CUDA library) in-tree with nvcc for sm_100a."""
+"""Builds ``libciar.so`` (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
+
+Every ``csrc/*.cu`` is compiled to an object of its own (in parallel, only when it or a header is
+newer than the object) and the objects are linked into the shared library.
+"""
 from __future__ import annotations
 
 import glob
 import os
 import shutil
 import subprocess
+from concurrent.futures import ThreadPoolExecutor
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libciar.so")
+OBJ_DIR = os.path.join(_PKG, "_build")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared",
+    "-Xcompiler", "-fPIC",
 ]
 
 
@@ -29,33 +35,62 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
+def _headers():
+    return glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) + \
+        glob.glob(os.path.join(INCLUDE, "*.h"))
+
+
 def is_stale() -> bool:
     if not os.path.exists(LIB_PATH):
         return True
     t = os.path.getmtime(LIB_PATH)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) + \
-        glob.glob(os.path.join(INCLUDE, "*.h"))
-    return any(os.path.getmtime(d) > t for d in deps)
+    return any(os.path.getmtime(d) > t for d in sources() + _headers())
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into libciar.so if it is missing or older than a source."""
-    if not force and not is_stale():
-        return LIB_PATH
-    tmp = LIB_PATH + ".tmp%d" % os.getpid()
+def _obj_of(src: str) -> str:
+    return os.path.join(OBJ_DIR, os.path.splitext(os.path.basename(src))[0] + ".o")
+
+
+def _compile(src: str, verbose: bool) -> str:
     cmd = [_nvcc()] + NVCC_FLAGS + ["-I", INCLUDE, "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += sources() + ["-o", tmp]
+    cmd += ["-c", src, "-o", _obj_of(src)]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+        raise RuntimeError("nvcc failed on %s:\n%s%s" % (os.path.basename(src), res.stdout, res.stderr))
+    return res.stderr
+
+
+def build_library(force: bool = False, verbose: bool = False) -> str:
+    """Compile what is missing or older than a source and link libciar.so."""
+    if not force and not is_stale():
+        return LIB_PATH
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    newest_header = max([os.path.getmtime(h) for h in _headers()] + [0.0])
+    todo = []
+    for src in sources():
+        obj = _obj_of(src)
+        if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), newest_header):
+            todo.append(src)
+    with ThreadPoolExecutor(max_workers=max(1, min(len(todo), os.cpu_count() or 4))) as pool:
+        logs = list(pool.map(lambda s: _compile(s, verbose), todo))
+    # objects of sources that no longer exist must not be linked
+    wanted = {_obj_of(s) for s in sources()}
+    for obj in glob.glob(os.path.join(OBJ_DIR, "*.o")):
+        if obj not in wanted:
+            os.remove(obj)
+    tmp = LIB_PATH + ".tmp%d" % os.getpid()
+    cmd = [_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a"] + sorted(wanted) + ["-o", tmp]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("link failed:\n" + res.stdout + res.stderr)
     os.replace(tmp, LIB_PATH)
     if verbose:
-        print(res.stderr)
+        print("\n".join(logs))
     return LIB_PATH
 
 
 if __name__ == "__main__":
     import sys
-    print(build_library(force=True, verbose="-v" in sys.argv))
+    print(build_library(force="-f" in sys.argv, verbose="-v" in sys.argv))

@@ -8,6 +8,9 @@ namespace ciar {
 
 namespace {
 std::atomic<int64_t> g_launches{0};
+// bound of the device-side waits (about a second of SM clocks) and the test hook that withholds one row's copy
+std::atomic<int64_t> g_wait_cycles{2000000000ll};
+std::atomic<int32_t> g_drop_cta{-1}, g_drop_k{-1};
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -68,6 +71,9 @@ void fill_quantify_args(QuantifyArgs &a, const ciar_logits_desc *d, const void *
     a.policy = p->policy;
     a.tau = p->tau;
     a.u_flag = p->u_flag;
+    a.wait_cycles = g_wait_cycles.load(std::memory_order_relaxed);
+    a.drop_cta = g_drop_cta.load(std::memory_order_relaxed);
+    a.drop_k = g_drop_k.load(std::memory_order_relaxed);
 }
 
 // Layout of the workspace: verify scratch first, then the per-step arrays of the decode loop.

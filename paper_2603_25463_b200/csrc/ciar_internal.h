@@ -18,6 +18,10 @@ struct QuantifyArgs {
     float tau;
     const float *u_flag;
     ciar_quantify_out out;  // indexed by logical row
+    // streaming kernels: bound of every device-side wait, in SM clocks, and (test hook, off when negative)
+    // the CTA and the place in its walk of one row whose copy is never issued
+    int64_t wait_cycles;
+    int32_t drop_cta, drop_k;
 };
 
 // Scratch of one verify launch, carved out of the caller's workspace.

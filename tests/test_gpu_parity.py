@@ -191,6 +191,132 @@ def test_quantify_streaming_rows_with_many_large_codes(ciar, dtype):
     assert rep.near_tie_flags <= 1
 
 
+def _sm_count():
+    return torch.cuda.get_device_properties(0).multi_processor_count
+
+
+def _edge_rows(v, g, with_many_large=True):
+    """The rows that exercise every special path of the streaming quantifiers, for a row of v codes: ordinary
+    rows of several sharpnesses, degenerate rows (one-hot, constant, near one-hot, two equal maxima far apart,
+    ties of the maximum, a long -inf stretch, a huge dynamic range, nearly uniform rows), rows with tens to
+    hundreds of codes above the exactly treated level, and unusable rows (NaN, no finite code, +inf)."""
+    rows, kinds = [], []
+    def add(kind, row):
+        rows.append(row); kinds.append(kind)
+    for scale in (8.0, 1.0, 3.0, 0.3, 0.05):
+        add("ordinary", torch.randn(v, generator=g) * scale)
+    one_hot = torch.full((v,), float("-inf")); one_hot[v // 3] = 2.5; add("one_hot", one_hot)
+    add("constant", torch.full((v,), -0.75))
+    near = torch.full((v,), -30.0); near[v - 9] = 20.0; add("near_one_hot", near)
+    two = torch.full((v,), float("-inf")); two[3] = 1.0; two[v - 400] = 1.0; add("two_hot", two)
+    ties = torch.zeros(v); ties[40:44] = 5.0; ties[v - 1] = 5.0; add("ties", ties)
+    holes = torch.randn(v, generator=g); holes[100:v // 2 + 600] = float("-inf"); add("holes", holes)
+    add("huge_range", torch.randn(v, generator=g) * 1e4)
+    add("flat_small", torch.randn(v, generator=g) * 1e-3)
+    add("flat_offset", 7.0 + torch.randn(v, generator=g) * 0.02)
+    if with_many_large:
+        for tops in (1, 40, 200, 650, 33, 31):
+            row = torch.randn(v, generator=g) * 0.5 - 6.0
+            row[torch.randperm(v, generator=g)[:tops]] = 5.0 + 0.01 * torch.randn(tops, generator=g)
+            add("tops%d" % tops, row)
+    nan_row = torch.randn(v, generator=g); nan_row[v - 2] = float("nan"); add("nan", nan_row)
+    add("no_finite", torch.full((v,), float("-inf")))
+    inf_row = torch.randn(v, generator=g); inf_row[9] = float("inf"); add("pos_inf", inf_row)
+    return torch.stack(rows), kinds
+
+
+def _tile(base, total, g):
+    """`total` rows drawn from `base` in a seeded shuffled order in which every kind of row follows every other."""
+    idx = torch.randint(0, base.shape[0], (total,), generator=g)
+    idx[:base.shape[0]] = torch.arange(base.shape[0])
+    return idx
+
+
+@pytest.mark.parametrize("dtype,v", [(torch.bfloat16, 16384), (torch.bfloat16, 8192), (torch.bfloat16, 5000),
+                                     (torch.bfloat16, 2048), (torch.float32, 16384), (torch.float32, 3000)])
+def test_quantify_streaming_edge_rows_many_per_cta(ciar, dtype, v):
+    """Every kind of special row next to every other inside one CTA's walk of the streaming quantifier: far more
+    rows than the persistent grid has CTAs, in a shuffled order, with radii on both sides of the series / direct
+    switch (and a NaN radius), so that the ring's stages, the slots the sweep warps fill, and the batches of the
+    finishing warps are reused many times by rows of different kinds."""
+    g = torch.Generator().manual_seed(v + (1 if dtype == torch.float32 else 0))
+    base, kinds = _edge_rows(v, g)
+    cap = _sm_count() * 2
+    total = 20 * cap + 7 if v <= 8192 else 16 * cap + 7
+    idx = _tile(base, total, g)
+    logits = base.to(dtype)[idx].contiguous()
+    assert logits.shape[0] > 16 * cap
+    rad_choices = torch.tensor([0.05, 1.0, 0.3, 0.9, 2.5, 0.0, 1.0000001, 7.0])
+    radius = rad_choices[torch.randint(0, len(rad_choices), (total,), generator=g)]
+    radius[total // 2] = float("nan")
+    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=radius, tau=1e-4)
+    ref, out, rep = pu.check_quantify(logits, prm)
+    st = out.row_status.cpu().numpy()
+    k = np.array(kinds, dtype=object)[idx.numpy()]
+    ok_radius = ~np.isnan(radius.numpy())
+    assert (st[(k == "nan") | (k == "pos_inf")] & oracle.ROW_NAN).all()
+    assert (st[k == "no_finite"] == oracle.ROW_NO_FINITE).all()
+    assert (st[(k == "ordinary") & ok_radius] == 0).all() and st[total // 2] & oracle.ROW_NAN
+    assert (out.argmax.cpu().numpy()[(k == "ties") & ok_radius] == 40).all()
+    print("near-tie flags: %d of %d rows" % (rep.near_tie_flags, total))
+    assert rep.near_tie_flags <= 4
+
+
+@pytest.mark.parametrize("raw", [False, True])
+@pytest.mark.parametrize("dtype,v", [(torch.bfloat16, 2048), (torch.bfloat16, 16384), (torch.float32, 4096)])
+def test_quantify_per_code_edge_rows_many_per_cta(ciar, dtype, v, raw):
+    """The per-code streaming quantifier on far more rows than its grid has CTAs: special rows of every kind in a
+    shuffled order, so that its parked-row batches fill and its stages are reused by rows of different kinds."""
+    g = torch.Generator().manual_seed(3 * v + int(raw))
+    base, kinds = _edge_rows(v, g, with_many_large=False)
+    cap = _sm_count()
+    total = 21 * cap + 5
+    idx = _tile(base, total, g)
+    logits = base.to(dtype)[idx].contiguous()
+    assert logits.shape[0] > 16 * cap
+    nb = 12  # a dozen radius rows, drawn like the logit rows
+    if raw:
+        rbase = torch.randn(nb, v, generator=g) * 1.5 - 1.0
+        rbase[1] = -12.0 + torch.randn(v, generator=g)
+        rbase[2] = 6.0 + torch.randn(v, generator=g)
+    else:
+        rbase = torch.rand(nb, v, generator=g) * 2.0
+        rbase[1] = torch.rand(v, generator=g) * 1e-3
+        rbase[2] = 4.0 + torch.rand(v, generator=g)
+        rbase[3] = torch.rand(v, generator=g) * 0.6
+    rbase[4] = 0.4
+    ridx = torch.randint(0, nb, (total,), generator=g)
+    ridx[idx == kinds.index("constant")] = 4  # constant row with constant radius: Sigma = 0
+    radius = rbase.to(dtype)[ridx].contiguous()
+    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_CODE, radius=radius, radius_is_raw=raw, r_max=2.5, tau=1e-4)
+    ref, out, rep = pu.check_quantify(logits, prm)
+    print("near-tie flags: %d of %d rows" % (rep.near_tie_flags, total))
+    assert rep.near_tie_flags <= 4
+
+
+@pytest.mark.parametrize("dtype,v", [(torch.bfloat16, 16392), (torch.bfloat16, 20480), (torch.float32, 17000)])
+def test_quantify_wide_edge_rows_many_per_cta(ciar, dtype, v):
+    """The chunked quantifier for rows that do not fit a stage, on far more rows than its grid has CTAs."""
+    g = torch.Generator().manual_seed(5 * v)
+    base, kinds = _edge_rows(v, g)
+    extra = []
+    late = torch.randn(v, generator=g); late[v - 3] = 30.0; extra.append(late)
+    rising = torch.randn(v, generator=g) + torch.linspace(0.0, 40.0, v); extra.append(rising)
+    ties = torch.zeros(v); ties[[16390, 300, v - 1, 9000]] = 5.0; extra.append(ties)
+    base = torch.cat([base, torch.stack(extra)])
+    cap = _sm_count()
+    total = 21 * cap + 3
+    idx = _tile(base, total, g)
+    logits = base.to(dtype)[idx].contiguous()
+    assert logits.shape[0] > 16 * cap
+    rad_choices = torch.tensor([0.05, 1.0, 0.3, 2.5, 0.9])
+    radius = rad_choices[torch.randint(0, len(rad_choices), (total,), generator=g)]
+    prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=radius, tau=1e-3)
+    ref, out, rep = pu.check_quantify(logits, prm)
+    print("near-tie flags: %d of %d rows" % (rep.near_tie_flags, total))
+    assert rep.near_tie_flags <= 4
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("v", [16392, 40000, 65536 + 4096])
 def test_quantify_wide_rows(ciar, v, dtype):
