@@ -244,6 +244,19 @@ ciar_status ciar_decode_step(const ciar_decode_state *state, const ciar_logits_d
                              const ciar_interval_params *params, const ciar_verify_params *vparams,
                              void *ws, size_t ws_bytes, void *stream);
 
+/*
+ * Test hook for the bounded device-side waits (the paper has no counterpart; not for production use).
+ * The streaming kernels wait for a row's bytes to land on chip with a bound of about a second of SM
+ * clocks; a wait that runs out ends the CTA's walk, and the rows it had not finished get
+ * CIAR_ROW_TIMEOUT in row_status (flag 1, scores NaN) while the call itself still returns CIAR_OK --
+ * no entry point returns CIAR_ERR_TIMEOUT; that code is reserved.  This hook makes such a wait run out
+ * without any fault: in every later ciar_quantify launch of the streaming quantifier, CTA `cta` never
+ * asks for the `row_in_walk`-th row of its walk (nothing is left in flight), and every wait is bounded
+ * by `wait_cycles` SM clocks.  cta < 0 switches the hook off; wait_cycles <= 0 restores the default bound.
+ * Host-side state, process-wide; returns CIAR_OK.
+ */
+ciar_status ciar_test_stall(int32_t cta, int32_t row_in_walk, int64_t wait_cycles);
+
 /* Human-readable name of a status code (host pointer to a static string). */
 const char *ciar_status_string(ciar_status s);
 

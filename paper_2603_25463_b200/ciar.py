@@ -18,7 +18,7 @@ F32, BF16 = 0, 1
 RADIUS_SCALAR, RADIUS_PER_ROW, RADIUS_PER_CODE = 0, 1, 2
 POLICY_INTERVAL, POLICY_ENTROPY, POLICY_MAXPROB, POLICY_RANDOM, POLICY_ALL = 0, 1, 2, 3, 4
 VERIFY_ANCHORED, VERIFY_PER_TOKEN, VERIFY_ALL = 0, 1, 2
-ROW_NAN, ROW_NO_FINITE, ROW_BAD_TOKEN = 1, 2, 4
+ROW_NAN, ROW_NO_FINITE, ROW_BAD_TOKEN, ROW_TIMEOUT = 1, 2, 4, 8
 MAX_WINDOW = 64
 
 _vp = ctypes.c_void_p
@@ -89,6 +89,8 @@ def load() -> ctypes.CDLL:
         lib.ciar_verify_static.restype = ctypes.c_int
         lib.ciar_verify_static.argtypes = [ctypes.POINTER(LogitsDesc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                            ctypes.POINTER(VerifyParamsC), ctypes.POINTER(VerifyOutC), _vp]
+        lib.ciar_test_stall.restype = ctypes.c_int
+        lib.ciar_test_stall.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int64]
         lib.ciar_decode_init.restype = ctypes.c_int
         lib.ciar_decode_init.argtypes = [ctypes.POINTER(DecodeStateC), ctypes.c_int32, _vp]
         lib.ciar_decode_step.restype = ctypes.c_int
@@ -109,6 +111,12 @@ def version() -> int:
 
 def launch_count() -> int:
     return int(load().ciar_launch_count())
+
+
+def stall_hook(cta: int, row_in_walk: int, wait_cycles: int) -> None:
+    """Test hook: CTA `cta` of the streaming quantifier never asks for the `row_in_walk`-th row of its walk and every
+    device-side wait is bounded by `wait_cycles` SM clocks (cta < 0: off; wait_cycles <= 0: default bound)."""
+    load().ciar_test_stall(int(cta), int(row_in_walk), int(wait_cycles))
 
 
 def workspace_bytes(rows: int, window: int) -> int:

@@ -144,6 +144,14 @@ const char *ciar_status_string(ciar_status s)
 
 int ciar_version(void) { return CIAR_VERSION; }
 
+ciar_status ciar_test_stall(int32_t cta, int32_t row_in_walk, int64_t wait_cycles)
+{
+    g_drop_cta.store(cta < 0 ? -1 : cta, std::memory_order_relaxed);
+    g_drop_k.store(cta < 0 ? -1 : row_in_walk, std::memory_order_relaxed);
+    g_wait_cycles.store(wait_cycles > 0 ? wait_cycles : 2000000000ll, std::memory_order_relaxed);
+    return CIAR_OK;
+}
+
 int64_t ciar_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 size_t ciar_workspace_bytes(int64_t rows, int32_t window)

@@ -48,7 +48,7 @@ __device__ __forceinline__ RadiusConst code_radius(const RowView<T> &, float rho
 {
     float r = rho;
     if (raw) r = (rho > 0.f) ? rho + log1pf(expf(-rho)) : log1pf(expf(rho));
-    r = fminf(r, r_max);
+    r = !(r > r_max) ? r : r_max;  // (a NaN radius stays NaN and marks the row)
     RadiusConst k;
     k.alpha = -expm1f(-r);
     k.beta = expm1f(r);
@@ -169,6 +169,30 @@ __global__ void __launch_bounds__(kThreads) quantify_kernel(QuantifyArgs a)
 
         // normalisation step and score, in double (every thread computes the same values)
         const double A = acc[0], B = acc[1], AA = acc[2], AB = acc[3], BB = acc[4];
+        if (PER_CODE && (!(A == A) || !(B == B))) {  // a NaN radius among the row's codes: the row is unusable
+            const float nanv = __int_as_float(0x7fc00000);
+            if (threadIdx.x == 0) {
+                if (o.row_max) o.row_max[lr] = nanv;
+                if (o.sum_exp) o.sum_exp[lr] = nanv;
+                if (o.lse) o.lse[lr] = nanv;
+                if (o.p_max) o.p_max[lr] = nanv;
+                if (o.entropy) o.entropy[lr] = nanv;
+                if (o.S_lo) o.S_lo[lr] = nanv;
+                if (o.S_up) o.S_up[lr] = nanv;
+                if (o.omega) o.omega[lr] = nanv;
+                if (o.sigma) o.sigma[lr] = nanv;
+                if (o.score) o.score[lr] = nanv;
+                if (o.argmax) o.argmax[lr] = -1;
+                if (o.flag) o.flag[lr] = 1;
+                if (o.row_status) o.row_status[lr] = (uint8_t)CIAR_ROW_NAN;
+            }
+            for (int32_t i = threadIdx.x; i < a.n; i += kThreads) {
+                if (dp) dp[i] = nanv;
+                if (dl) dl[i] = nanv;
+                if (du) du[i] = nanv;
+            }
+            continue;
+        }
         const double S_lo = B, S_up = A + B;
         double k_lo = 1.0, k_up = 1.0;
         if (S_lo > 0.0 && (double)a.lo_cap / S_lo < 1.0) k_lo = (double)a.lo_cap / S_lo;

@@ -254,6 +254,10 @@ __global__ void __launch_bounds__(kPcThreads, 1) quantify_percode_kernel(const _
             const PcTotals tt = row_totals(p, lane, p.m, p.nmax, p.dominant);
             const double dev = group_sum_d(p.dev, lane);
             if (lane != 0) return;
+            if (!(tt.A == tt.A) || !(tt.B == tt.B)) {  // a NaN radius among the row's codes (it went through every sum)
+                write_unusable(o, p.lr, CIAR_ROW_NAN);
+                return;
+            }
             const PcScales sc = row_scales(tt, a.lo_cap, a.hi_cap, nn);
             double var = (sc.k_up * sc.k_up * tt.AA + 2.0 * sc.k_up * sc.g * tt.AB + sc.g * sc.g * tt.BB) / nn - sc.mu * sc.mu;
             if (p.low_cv) var = dev / nn;

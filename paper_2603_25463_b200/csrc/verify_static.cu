@@ -1,5 +1,7 @@
 // ciar_verify_static: the cloud-side verification for callers that have no way to hand over a
 // workspace.  The scratch lives in a fixed array inside the library image instead.
+#include <atomic>
+
 #include "ciar_internal.h"
 
 namespace {
@@ -12,18 +14,19 @@ static __device__ __align__(256) unsigned char g_verify_scratch[CIAR_STATIC_SCRA
 // that device current.
 cudaError_t scratch_address(void **out)
 {
-    static void *cached[64] = {};
+    // (two host threads making the first call on a device at once both look the address up and store the same value)
+    static std::atomic<void *> cached[64] = {};
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (cached[dev] == nullptr) {
-        void *p = nullptr;
+    void *p = cached[dev].load(std::memory_order_acquire);
+    if (p == nullptr) {
         err = cudaGetSymbolAddress(&p, g_verify_scratch);
         if (err != cudaSuccess) return err;
-        cached[dev] = p;
+        cached[dev].store(p, std::memory_order_release);
     }
-    *out = cached[dev];
+    *out = p;
     return cudaSuccess;
 }
 

@@ -58,6 +58,30 @@ def assert_close(name, got, want, rep: Optional[Report] = None, rtol=RTOL, atol=
                              (name, bad.sum(), bad.size, i, got.ravel()[i], want.ravel()[i]))
 
 
+GUARD = 64  # canary elements on either side of every output array
+
+
+class Guarded:
+    """Puts every tensor of an output object (QuantifyOut, VerifyOut) between two runs of a byte pattern inside a larger
+    buffer; check() says whether a kernel wrote outside any of them."""
+
+    def __init__(self, out):
+        self.out, self.bufs = out, []
+        for name, t in list(vars(out).items()):
+            if not isinstance(t, torch.Tensor):
+                continue
+            n = t.numel()
+            buf = torch.empty(n + 2 * GUARD, dtype=t.dtype, device=t.device)
+            buf.view(torch.uint8).fill_(0xA5)
+            setattr(out, name, buf[GUARD:GUARD + n].view(t.shape))
+            self.bufs.append((name, buf, n))
+
+    def check(self):
+        for name, buf, n in self.bufs:
+            edge = torch.cat([buf[:GUARD], buf[GUARD + n:]]).view(torch.uint8)
+            assert bool((edge == 0xA5).all()), "a kernel wrote outside the output array %s" % name
+
+
 def to_ciar_params(p: oracle.IntervalParams, device) -> ciar.IntervalParams:
     def dev(x, dtype=None):
         if x is None:
@@ -85,11 +109,13 @@ def check_quantify(logits_cpu: torch.Tensor, params: oracle.IntervalParams, vali
     ref = oracle.quantify(logits_cpu, params, valid_begin, n, dense=dense, threads=threads)
     ld = logits_cpu.to(device) if logits_dev is None else logits_dev
     out = ciar.QuantifyOut.allocate(rows, device, dense_width=n if dense else 0)
+    guard = Guarded(out)
     gp = to_ciar_params(params, device)
     if radius_dev is not None:
         gp.radius = radius_dev
     ciar.quantify(ld, gp, out, valid_begin, n)
     torch.cuda.synchronize()
+    guard.check()
     rep = Report(rows=rows)
     for name in Q_FLOAT_FIELDS:
         assert_close(name, getattr(out, name).cpu().numpy(), getattr(ref, name), rep)
@@ -120,12 +146,14 @@ def check_verify(draft_cpu, target_cpu, tokens, flag, u_accept, u_resample, wind
     td = target_cpu.to(device) if target_dev is None else target_dev
     as_dev = lambda x, dt: None if x is None else torch.as_tensor(np.asarray(x.cpu() if isinstance(x, torch.Tensor) else x)).to(dt).to(device)
     out = ciar.VerifyOut.allocate(rows, window, device)
+    guard = Guarded(out)
     ws = ciar.alloc_workspace(rows, window, device)
     rm, se = draft_stats if draft_stats is not None else (None, None)
     ciar.verify(dd, td, as_dev(tokens, torch.int32), as_dev(flag, torch.uint8), rm, se,
                 as_dev(u_accept, torch.float32), as_dev(u_resample, torch.float32), window, mode, out, ws,
                 valid_begin, n)
     torch.cuda.synchronize()
+    guard.check()
     rep = Report(rows=rows, windows=rows // window)
     assert np.array_equal(out.row_status.cpu().numpy(), ref.row_status), "verify row_status"
     assert np.array_equal(out.first_flag.cpu().numpy(), ref.first_flag), "first_flag"

@@ -56,6 +56,39 @@ def test_verify_static_matches_verify_on_two_calls_in_a_row(ciar_lib):
         assert (want.accepted_len < window).any()  # some window was rejected, so the resampling path ran
 
 
+def test_verify_static_streaming_path_on_used_scratch_matches_verify_and_oracle(ciar_lib):
+    """The path production takes (draft statistics from ciar_quantify, rows of 2048 codes and more: plan, accept sweep and
+    window kernels working out of the scratch) through the shared array, twice in a row with different row counts and
+    windows, so that the second call finds the first one's counters and lists where it reads.  Checked against
+    ciar_verify with an ordinary workspace and against the CPU oracle."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import oracle
+    import parity_util as pu
+    ciar = ciar_lib
+    cases = [(8 * 40, 4096, 8, 21, torch.bfloat16, ciar.VERIFY_ANCHORED), (16 * 9, 2048, 16, 22, torch.float32, ciar.VERIFY_ALL),
+             (4 * 50, 2056, 4, 23, torch.bfloat16, ciar.VERIFY_PER_TOKEN)]
+    for rows, v, window, seed, dtype, mode in cases:
+        draft, target, tokens, flag, ua, ur = _case(rows, v, window, seed, dtype)
+        qo = ciar.QuantifyOut.allocate(rows, "cuda")
+        ciar.quantify(draft, ciar.IntervalParams(r_scalar=0.2, tau=1e-4), qo)
+        want = ciar.VerifyOut.allocate(rows, window, "cuda")
+        ws = ciar.alloc_workspace(rows, window, "cuda")
+        ciar.verify(draft, target, tokens, flag, qo.row_max, qo.sum_exp, ua, ur, window, mode, want, ws)
+        got = ciar.VerifyOut.allocate(rows, window, "cuda")
+        ciar.verify_static(draft, target, tokens, flag, qo.row_max, qo.sum_exp, ua, ur, window, mode, got)
+        torch.cuda.synchronize()
+        _compare(ciar, got, want)
+        ref = oracle.verify(draft.cpu(), target.cpu(), tokens.cpu().numpy(), flag.cpu().numpy(), ua.cpu().numpy(),
+                            ur.cpu().numpy(), window, mode)
+        win_ok = ~((ref.accept_margin < pu.NEAR_TIE).reshape(-1, window).any(1) | (ref.resample_margin < pu.NEAR_TIE))
+        assert np.array_equal(got.first_flag.cpu().numpy(), ref.first_flag)
+        assert np.array_equal(got.accepted_len.cpu().numpy()[win_ok], ref.accepted_len[win_ok])
+        assert np.array_equal(got.resampled_token.cpu().numpy()[win_ok], ref.resampled_token[win_ok])
+        assert np.array_equal(got.accept.cpu().numpy()[np.repeat(win_ok, window)], ref.accept[np.repeat(win_ok, window)])
+        assert win_ok.sum() >= 0.9 * len(win_ok) and (ref.accepted_len < window).any()
+
+
 def test_verify_static_refuses_more_rows_than_its_scratch_serves(ciar_lib):
     if not torch.cuda.is_available():
         pytest.skip("needs a CUDA device")
