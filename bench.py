@@ -50,24 +50,28 @@ class ClockSampler:
 
     def __init__(self, device_index: int):
         self.proc = None
+        self.why = None
         self.path = "/tmp/ciar_clocks_%d_%d.csv" % (os.getpid(), device_index)
         try:
             uuid = str(torch.cuda.get_device_properties(device_index).uuid)
             sel = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
         except Exception:
             sel = str(device_index)
-        self.cmd = ["nvidia-smi", "-i", sel, "--query-gpu=" + CLOCK_QUERY, "--format=csv,noheader,nounits", "-lms", "100"]
+        self.cmd = ["nvidia-smi", "-i", sel, "--query-gpu=" + CLOCK_QUERY, "--format=csv,noheader,nounits", "-lms", "50"]
 
     def start(self):
         try:
             self.out = open(self.path, "w")
-            self.proc = subprocess.Popen(self.cmd, stdout=self.out, stderr=subprocess.DEVNULL)
-        except Exception:
+            self.err = open(self.path + ".err", "w")
+            self.proc = subprocess.Popen(self.cmd, stdout=self.out, stderr=self.err)
+        except Exception as e:
             self.proc = None
+            self.why = "nvidia-smi could not be started: %r" % (e,)
 
     def stop(self):
         res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
+            res["note"] = self.why
             return res
         self.proc.terminate()
         try:
@@ -75,6 +79,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         self.out.close()
+        self.err.close()
         sm, mx, reasons = [], [], set()
         try:
             for line in open(self.path):
@@ -93,6 +98,15 @@ class ClockSampler:
             pass
         if sm:
             res.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        else:
+            try:
+                res["note"] = "no samples: " + open(self.path + ".err").read().strip()[:200]
+            except Exception:
+                res["note"] = "no samples"
+        try:
+            os.remove(self.path + ".err")
+        except Exception:
+            pass
         return res
 
 
@@ -162,6 +176,96 @@ class Step:
         return sent, resampled, flagged
 
 
+def timed_steps(ciar, step, K, warm, world, dev, roll_s=0.8):
+    """`warm` untimed steps, then K timed steps with CUDA events around every kernel of every step.  nvidia-smi samples the
+    clocks from before the first untimed step to after the last: the timed region is bracketed by about `roll_s` seconds
+    of the same steps on either side, so that the samples are taken under this very load even when K steps take a few
+    milliseconds.  Returns (total ms max over ranks, mean quantify ms, mean verify ms, clocks, launches in the timed region)."""
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    t0 = time.perf_counter()
+    for _ in range(warm):
+        step()
+    torch.cuda.synchronize()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s.record(); step(); e.record(); torch.cuda.synchronize()
+    est_ms = max(1e-3, s.elapsed_time(e))
+    roll = int(min(20000, max(0, roll_s * 1e3 / est_ms)))
+
+    def untimed(n):
+        for i in range(n):
+            step()
+            if i % 256 == 255:
+                torch.cuda.synchronize()  # keeps the launch queue short
+        torch.cuda.synchronize()
+    untimed(roll)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    launches0 = ciar.launch_count()
+    barrier(world)
+    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for k in range(K):
+        ev[k][0].record()
+        step.quantify()
+        ev[k][1].record()
+        step.verify()
+        ev[k][2].record()
+    t_end.record()
+    barrier(world)
+    launches = ciar.launch_count() - launches0
+    untimed(roll)
+    clocks = sampler.stop()
+    clocks["sampled_s"] = round(time.perf_counter() - t0, 2)
+    total_ms = max_over_ranks(t_start.elapsed_time(t_end), world)
+    q_ms = float(np.mean([ev[k][0].elapsed_time(ev[k][1]) for k in range(K)]))
+    v_ms = float(np.mean([ev[k][1].elapsed_time(ev[k][2]) for k in range(K)]))
+    clocks["time_x_mhz"] = None if clocks["sm_mhz"] is None else {"quantify": q_ms * clocks["sm_mhz"], "verify": v_ms * clocks["sm_mhz"]}
+    return total_ms, q_ms, v_ms, clocks, launches
+
+
+def config_of(name, wl, rows, radius):
+    """The workload as both arms name it."""
+    return {"workload": name, "rows_per_gpu": rows, "vocab": wl.vocab, "valid_codes": wl.n_valid, "logits": wl.dtype,
+            "window": wl.window, "verify_mode": "anchored", "radius": radius, "tau": wl.tau,
+            "l2": "inputs (%.0f MB) larger than L2; no flush" % (2 * rows * wl.n_valid * wl.elem_bytes / 1e6)}
+
+
+def kernel_names(wl, per_code):
+    wide = wl.n_valid > 16384  # rows that do not fit a stage take the chunked kernels
+    q = "quantify_percode_kernel" if per_code else ("quantify_wide_kernel" if wide else "quantify_stream_kernel")
+    return q, ("verify_plan+accept_wide+window" if wide else "verify_plan+accept+window")
+
+
+def workload_report(wl, rows, per_code, q_ms, v_ms, ms_per_step, sent, resampled, peak):
+    """Algorithmic bytes of one step and what they make of the measured times."""
+    row_bytes = wl.n_valid * wl.elem_bytes
+    q_bytes = rows * row_bytes * (2 if per_code else 1) + rows * 48  # a per-code radius row is as wide as its logit row
+    v_bytes = sent * row_bytes + resampled * 2 * row_bytes + rows * 16 + (rows // wl.window) * 16
+    q_name, v_name = kernel_names(wl, per_code)
+    q_gbs, v_gbs = q_bytes / (q_ms * 1e-3) / 1e9, v_bytes / (v_ms * 1e-3) / 1e9
+    return {q_name: {"ms": q_ms, "algorithmic_bytes": int(q_bytes), "GB/s": q_gbs, "frac": q_gbs / peak},
+            v_name: {"ms": v_ms, "algorithmic_bytes": int(v_bytes), "GB/s": v_gbs, "frac": v_gbs / peak},
+            "step_GB/s": (q_bytes + v_bytes) / (ms_per_step * 1e-3) / 1e9}
+
+
+def side_workload(ciar, name, steps, dev, peak):
+    """One of the other large-batch workloads, measured like the main one (device-resident, CUDA events, clocks sampled)."""
+    wl = synth.WORKLOADS[name]
+    inp = synth.make_inputs(wl, device=dev)
+    step = Step(ciar, wl, inp, False)
+    total_ms, q_ms, v_ms, clocks, _ = timed_steps(ciar, step, steps, 3, 1, dev, roll_s=0.6)
+    sent, resampled, flagged = step.traffic_model()
+    rep = workload_report(wl, step.rows, False, q_ms, v_ms, total_ms / steps, sent, resampled, peak)
+    rep.update({"rows": step.rows, "valid_codes": wl.n_valid, "logits": wl.dtype, "window": wl.window, "steps": steps,
+                "ms_per_step": total_ms / steps, "tokens/s": step.rows * steps / (total_ms * 1e-3),
+                "cloud_flag_fraction": flagged, "sent_fraction": sent / step.rows,
+                "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples")},
+                "l2": "inputs (%.0f MB) larger than L2; no flush" % (2 * step.rows * wl.n_valid * wl.elem_bytes / 1e6)})
+    del step, inp
+    torch.cuda.empty_cache()
+    return rep
+
+
 def run_ours(args):
     from paper_2603_25463_b200 import ciar
     rank, world, local = dist_setup(args.gpus)
@@ -176,33 +280,10 @@ def run_ours(args):
     rows = step.rows
     row_bytes = wl.n_valid * wl.elem_bytes
 
-    for _ in range(max(3, args.warmup)):
-        step()
-    torch.cuda.synchronize()
-    sent, resampled, flagged = step.traffic_model()
-
-    # ---- device-resident timing: K steps, events around every kernel of every step
+    warm = max(3, args.warmup)
+    total_ms, q_ms, v_ms, clocks, launches = timed_steps(ciar, step, args.steps, warm, world, dev)
     K = args.steps
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    sampler = ClockSampler(dev.index or 0)
-    launches0 = ciar.launch_count()
-    sampler.start()
-    barrier(world)
-    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    for k in range(K):
-        ev[k][0].record()
-        step.quantify()
-        ev[k][1].record()
-        step.verify()
-        ev[k][2].record()
-    t_end.record()
-    barrier(world)
-    clocks = sampler.stop()
-    launches = ciar.launch_count() - launches0
-    total_ms = max_over_ranks(t_start.elapsed_time(t_end), world)
-    q_ms = float(np.mean([ev[k][0].elapsed_time(ev[k][1]) for k in range(K)]))
-    v_ms = float(np.mean([ev[k][1].elapsed_time(ev[k][2]) for k in range(K)]))
+    sent, resampled, flagged = step.traffic_model()
     ms_per_step = total_ms / K
     value = world * rows * K / (total_ms * 1e-3)
 
@@ -243,26 +324,26 @@ def run_ours(args):
     if rank != 0:
         return
     peak, peak_kind = measured_peak()
-    q_bytes = rows * row_bytes * (2 if per_code else 1) + rows * 48  # a per-code radius row is as wide as its logit row
-    v_bytes = sent * row_bytes + resampled * 2 * row_bytes + rows * 16 + (rows // wl.window) * 16
-    q_gbs = q_bytes / (q_ms * 1e-3) / 1e9
-    v_gbs = v_bytes / (v_ms * 1e-3) / 1e9
-    wide = wl.n_valid > 16384  # rows that do not fit on chip take the two-pass / chunked kernels
-    q_name = "quantify_wide_kernel" if wide else "quantify_stream_kernel"
-    if per_code:
-        q_name = "quantify_percode_kernel"
-    v_name = "verify_plan+accept_wide+window" if wide else "verify_plan+accept+window"
+    kernels = workload_report(wl, rows, per_code, q_ms, v_ms, ms_per_step, sent, resampled, peak)
+    q_name, v_name = kernel_names(wl, per_code)
     dominant = q_name if q_ms >= v_ms else v_name
-    dom_gbs = q_gbs if q_ms >= v_ms else v_gbs
+    dom_gbs = kernels[dominant]["GB/s"]
     traffic = None if args.images else load_traffic(dominant, args.workload)  # the captures are of full batches
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
                 "frac": dom_gbs / peak, "peak_kind": "of " + peak_kind, "traffic": traffic,
                 "frac_of_nominal_8TBs": dom_gbs / NOMINAL_HBM_GBS,
-                "kernels": {q_name: {"ms": q_ms, "algorithmic_bytes": int(q_bytes), "GB/s": q_gbs,
-                                                "frac": q_gbs / peak},
-                            v_name: {"ms": v_ms, "algorithmic_bytes": int(v_bytes), "GB/s": v_gbs,
-                                              "frac": v_gbs / peak}},
-                "step_GB/s": (q_bytes + v_bytes) / (ms_per_step * 1e-3) / 1e9}
+                "kernels": {q_name: kernels[q_name], v_name: kernels[v_name]}, "step_GB/s": kernels["step_GB/s"]}
+    # the other large-batch workloads, each with its own kernel times, bytes and fractions (single GPU, default run)
+    per_workload = None
+    if world == 1 and args.side_workloads and not args.images and args.workload == "llamagen384" and not per_code:
+        del step, inp
+        torch.cuda.empty_cache()
+        per_workload = {}
+        for name, steps in (("anole", 200), ("largevocab", 5)):
+            try:
+                per_workload[name] = side_workload(ciar, name, steps, dev, peak)
+            except torch.cuda.OutOfMemoryError as e:
+                per_workload[name] = {"skipped": "not enough free device memory: %s" % str(e)[:80]}
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         cpu = cpu_oracle_baseline(synth.WORKLOADS[args.workload], sample_rows=args.cpu_rows)
@@ -270,13 +351,11 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "rows_per_gpu": rows, "vocab": wl.vocab, "valid_codes": wl.n_valid,
-                   "logits": wl.dtype, "window": wl.window, "verify_mode": "anchored", "radius": args.radius,
-                   "tau": wl.tau, "l2": "inputs (%.0f MB) larger than L2; no flush" % (2 * rows * row_bytes / 1e6)},
-        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                   "samples": clocks["samples"]},
+        "config": config_of(args.workload, wl, rows, args.radius),
+        "clocks": clocks,
         "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
         "cloud_flag_fraction": flagged, "sent_fraction": sent / rows, "resampled_windows": resampled,
+        "per_workload": per_workload,
     }
     print(json.dumps(line))
 
@@ -380,16 +459,28 @@ def run_decode(args):
         loop(False)  # warm-up of the replays
         torch.cuda.synchronize()
     sampler = ClockSampler(dev.index or 0)
-    launches0 = ciar.launch_count()
     sampler.start()
+    # whole untimed generations on either side of the timed one, so that the clock samples are taken under this load
+    w0 = time.perf_counter()
+    loop(False)
+    torch.cuda.synchronize()
+    n_roll = int(min(200, max(1, 0.8 / max(1e-3, time.perf_counter() - w0))))
+    for _ in range(n_roll):
+        loop(False)
+    torch.cuda.synchronize()
+    launches0 = ciar.launch_count()
     barrier(world)
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     steps, events = loop(True)
     t1.record()
     barrier(world)
+    launches_timed = ciar.launch_count() - launches0
+    for _ in range(n_roll):
+        loop(False)
+    torch.cuda.synchronize()
     clocks = sampler.stop()
-    launches = ciar.launch_count() - launches0
+    launches = launches_timed
     if graph is not None:
         launches = steps * launches_per_step  # replays do not pass through the library's counter
     total_ms = max_over_ranks(t0.elapsed_time(t1), world)
@@ -407,8 +498,7 @@ def run_decode(args):
                    "window": wl.window, "verify_mode": "anchored", "radius": args.radius, "tau": wl.tau,
                    "launch": "cuda graph replay" if graph is not None else "direct",
                    "l2": "pools of %.1f GB, rows touched once" % ((3 if per_code else 2) * req * seq * wl.vocab * wl.elem_bytes / 1e9)},
-        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                   "samples": clocks["samples"]},
+        "clocks": clocks,
         "gpu_launches": int(launches),
         "step_latency_us": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)),
                             "max": float(lat.max()), "timed_with": "CUDA events around every ciar_decode_step"},
@@ -425,7 +515,7 @@ def run_reference(args):
     import oracle
     wl = synth.WORKLOADS[args.workload]
     steps = max(1, min(args.steps, 20))
-    warm = max(1, min(args.warmup, 2))
+    warm = max(3, min(args.warmup, 5))
     inp = synth.make_inputs(wl, device="cpu", row_limit=args.cpu_rows)
     rows = inp.draft.shape[0]
     prm = oracle.IntervalParams(radius_mode=oracle.RADIUS_PER_ROW, radius=inp.radius_row, tau=wl.tau)
@@ -447,8 +537,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": steps,
         "warmup": warm, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "rows_per_step": rows, "vocab": wl.vocab, "valid_codes": wl.n_valid,
-                   "logits": wl.dtype, "window": wl.window, "verify_mode": "anchored", "radius": "per_row"},
+        "config": config_of(args.workload, wl, rows, "per_row"),
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -471,6 +560,8 @@ def main():
                     help="decode workload: replay each step from a CUDA graph (default) or launch it directly")
     ap.add_argument("--radius", default="per_row", choices=["per_row", "per_code"],
                     help="interval radius: one per row (default) or one raw value per code, a tensor as large as the logits")
+    ap.add_argument("--side-workloads", action=argparse.BooleanOptionalAction, default=True,
+                    help="default run on one GPU: also measure the anole and largevocab workloads (per_workload block)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

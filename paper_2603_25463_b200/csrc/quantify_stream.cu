@@ -84,35 +84,6 @@ __host__ __device__ constexpr int stages_for(int stage_bytes, int nfin, int wpr)
     return s > kMaxStages ? kMaxStages : s;
 }
 
-__device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
-}
-
-template <bool SLEEP>
-__device__ __noinline__ bool wait_phase_slow(unsigned long long *bar, uint32_t parity, volatile int *abort_flag, long long limit)
-{
-    const long long t0 = clock64();
-    for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (SLEEP) __nanosleep(40);
-        if (*abort_flag) return false;
-        if (clock64() - t0 > limit) {
-            *abort_flag = 1;
-            return false;
-        }
-    }
-}
-
-// Waits for the phase of the given parity; gives up (and tells everybody) after about `limit` clocks.
-// SLEEP: the wait is for data that may take a while (a row in flight); the warp naps between polls.
-template <bool SLEEP = true>
-__device__ __forceinline__ bool wait_phase(unsigned long long *bar, uint32_t parity, int *abort_flag, long long limit)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    return wait_phase_slow<SLEEP>(bar, parity, abort_flag, limit);
-}
-
 // Sums four values over the warp with six shuffles: on return lanes 0..7 hold the sum of v0, 8..15 of v1,
 // 16..23 of v2, 24..31 of v3.
 __device__ __forceinline__ float warp_sum4(float v0, float v1, float v2, float v3, int lane)

@@ -53,6 +53,36 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, uint3
     return false;
 }
 
+// One plain arrival.
+__device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+template <bool SLEEP>
+__device__ __noinline__ bool wait_phase_slow(unsigned long long *bar, uint32_t parity, volatile int *abort_flag, long long limit)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (SLEEP) __nanosleep(40);
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limit) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+// Waits for the phase of the given parity; gives up (and tells everybody) after about `limit` clocks.
+// SLEEP: the wait is for data that may take a while (a row in flight); the warp naps between polls.
+template <bool SLEEP = true>
+__device__ __forceinline__ bool wait_phase(unsigned long long *bar, uint32_t parity, int *abort_flag, long long limit)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return wait_phase_slow<SLEEP>(bar, parity, abort_flag, limit);
+}
+
 // Bulk copy of `bytes` (a multiple of 16; both addresses 16-byte aligned) from global to this
 // CTA's shared memory; completion is signalled on `bar` as `bytes` of transaction count.
 __device__ __forceinline__ void bulk_copy_g2s(void *dst_smem, const void *src_gmem, uint32_t bytes, unsigned long long *bar)
