@@ -129,32 +129,14 @@ struct VShared {
     VParked park[kVPark];
 };
 
-// The accept test of one tested row, by one warp: u * p_x < q_x in double, p and q the draft's
-// and the target's probability of the drafted token.
+// The accept test of one tested row from the two rows' softmax statistics, by one thread: u * p_x < q_x in double, p and q
+// the draft's and the target's probability of the drafted token.  status: what is already known to be wrong with the row.
 template <typename T>
-__device__ __noinline__ void accept_row(const VerifyArgs &a, const VParked &pk, int lane)
+__device__ __forceinline__ void accept_decide(const VerifyArgs &a, int64_t lr, int64_t pr, float mq, double zq, float mp, double zp,
+                                              int status)
 {
-    const int64_t lr = pk.lr;
-    int64_t pr;
-    map_row(a.rm, lr, pr);
     const T *drow = reinterpret_cast<const T *>(a.draft) + pr * a.row_stride + a.vb;
     const T *trow = reinterpret_cast<const T *>(a.target) + pr * a.row_stride + a.vb;
-    // target statistics from the sweeps
-    double zq = lane < kVWarps ? (double)pk.wz[lane] : 0.0;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) zq += __shfl_xor_sync(0xffffffffu, zq, o);
-    zq += (double)pk.nmax * (double)pk.e0;
-    float mq = pk.m;
-    // the exponent used was c * log2e_f - fl(m * log2e_f): take the common offset out again
-    const double off = (double)mq * (double)kLog2e - (double)(mq * kLog2e);
-    zq *= exp2(-off);
-    int status = 0;
-    if (!(mq > -INFINITY) || !(zq > 0.0) || !(zq < INFINITY)) status |= warp_row_stats(trow, a.n, lane, mq, zq);
-    // draft statistics from the quantifier; unusable ones are recomputed to learn what is wrong with the row
-    float mp = a.draft_row_max[lr];
-    double zp = (double)a.draft_sum_exp[lr];
-    if (!(zp > 0.0) || !(zp < INFINITY) || !(mp == mp)) status |= warp_row_stats(drow, a.n, lane, mp, zp);
-    if (lane != 0) return;
     const int32_t x = a.tokens[pr];
     const bool bad_token = (x < 0 || x >= a.vocab);
     if (bad_token) status |= CIAR_ROW_BAD_TOKEN;
@@ -186,164 +168,253 @@ __device__ __noinline__ void accept_row(const VerifyArgs &a, const VParked &pk, 
     if (a.out.row_status) a.out.row_status[lr] = (uint8_t)status;
 }
 
-template <typename T, int JV, bool FULL>
-__global__ void __launch_bounds__(kVThreads, 2) verify_accept_kernel(const __grid_constant__ VerifyArgs a)
+// The accept test of one tested row whose target statistics are parked, by one warp.
+template <typename T>
+__device__ __noinline__ void accept_row(const VerifyArgs &a, const VParked &pk, int lane)
+{
+    const int64_t lr = pk.lr;
+    int64_t pr;
+    map_row(a.rm, lr, pr);
+    const T *drow = reinterpret_cast<const T *>(a.draft) + pr * a.row_stride + a.vb;
+    const T *trow = reinterpret_cast<const T *>(a.target) + pr * a.row_stride + a.vb;
+    // target statistics from the sweeps
+    double zq = lane < kVWarps ? (double)pk.wz[lane] : 0.0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) zq += __shfl_xor_sync(0xffffffffu, zq, o);
+    zq += (double)pk.nmax * (double)pk.e0;
+    float mq = pk.m;
+    // the exponent used was c * log2e_f - fl(m * log2e_f): take the common offset out again
+    const double off = (double)mq * (double)kLog2e - (double)(mq * kLog2e);
+    zq *= exp2(-off);
+    int status = 0;
+    if (!(mq > -INFINITY) || !(zq > 0.0) || !(zq < INFINITY)) status |= warp_row_stats(trow, a.n, lane, mq, zq);
+    // draft statistics from the quantifier; unusable ones are recomputed to learn what is wrong with the row
+    float mp = a.draft_row_max[lr];
+    double zp = (double)a.draft_sum_exp[lr];
+    if (!(zp > 0.0) || !(zp < INFINITY) || !(mp == mp)) status |= warp_row_stats(drow, a.n, lane, mp, zp);
+    if (lane != 0) return;
+    accept_decide<T>(a, lr, pr, mq, zq, mp, zp, status);
+}
+
+// ---- accept, rows that fit a shared-memory stage.  One persistent CTA per SM walks its share of the list; its warps
+// have three roles that meet on mbarriers only: a producer thread that copies each target row into the next free stage
+// with one bulk (TMA) copy, several rows ahead; 16 sweep warps, in groups of WPR warps that share a row (the groups take
+// alternate rows), each warp summing exp(t - its own share's maximum) over its share; and a few finishing warps that bring
+// the warps' sums to the row maximum, join them, hand the stage back and file the row; every 32 rows a finishing warp does
+// the accept tests of its batch, a row per lane (the drafted token's two logits come from global memory).
+constexpr int kACW = 16;     // sweep warps
+constexpr int kAJV = 8;      // 16-byte vectors of a row one lane owns (at most)
+constexpr int kAFin = 3;     // finishing warps
+constexpr int kABatch = 32;  // rows per batch of accept tests
+constexpr int kAMaxStages = 16;
+constexpr int kASmem = 227 * 1024;
+
+template <int WPR>
+struct ASlot {
+    unsigned long long full, swept, empty;  // the row has landed / every warp has published its sum / the stage may be refilled
+    int64_t lr;                             // logical row (-1: nothing to do)
+    float wmax[WPR], wz[WPR];               // per warp: maximum of its share, sum of exp(t - that maximum)
+};
+
+struct ABatch {
+    int64_t lr[kABatch];
+    float m[kABatch], z[kABatch];  // row maximum, sum of exp(t - m) as computed (offset of the exponent still in it)
+};
+
+template <int S, int WPR>
+struct AControl {
+    ASlot<WPR> slot[S];
+    int abort, issued;
+    int fin_next[kAFin];
+    ABatch batch[kAFin];
+};
+
+__host__ __device__ constexpr int accept_stages(int stage_bytes)
+{
+    int s = (kASmem - 4096) / (stage_bytes + 256);
+    return s > kAMaxStages ? kAMaxStages : s;
+}
+
+// The accept tests of a batch, a row per lane; rows whose statistics came out unusable are then redone one by one by the
+// whole warp, which learns from the rows themselves what is wrong with them.
+template <typename T>
+__device__ __noinline__ void accept_batch(const VerifyArgs &a, const ABatch &bt, int count, int lane)
+{
+    int64_t lr = 0, pr = 0;
+    bool slow = false;
+    if (lane < count) {
+        lr = bt.lr[lane];
+        map_row(a.rm, lr, pr);
+        float mq = bt.m[lane];
+        // the exponent used was c * log2e_f - fl(m * log2e_f): take the common offset out again
+        const double off = (double)mq * (double)kLog2e - (double)(mq * kLog2e);
+        const double w2 = -off * kLn2D;
+        const double zq = (double)bt.z[lane] * (1.0 + w2 * (1.0 + 0.5 * w2));  // 2^-off, |off| far below 1e-4
+        const float mp = a.draft_row_max[lr];
+        const double zp = (double)a.draft_sum_exp[lr];
+        slow = !(mq > -INFINITY) || !(mq < INFINITY) || !(zq > 0.0) || !(zq < (double)INFINITY) || !(zp > 0.0) ||
+               !(zp < (double)INFINITY) || !(mp == mp);
+        if (!slow) accept_decide<T>(a, lr, pr, mq, zq, mp, zp, 0);
+    }
+    for (unsigned todo = __ballot_sync(0xffffffffu, slow); todo != 0; todo &= todo - 1) {
+        const int h = __ffs((int)todo) - 1;
+        const int64_t lr_h = __shfl_sync(0xffffffffu, lr, h), pr_h = __shfl_sync(0xffffffffu, pr, h);
+        const T *drow = reinterpret_cast<const T *>(a.draft) + pr_h * a.row_stride + a.vb;
+        const T *trow = reinterpret_cast<const T *>(a.target) + pr_h * a.row_stride + a.vb;
+        float mq, mp = a.draft_row_max[lr_h];
+        double zq, zp = (double)a.draft_sum_exp[lr_h];
+        int status = warp_row_stats(trow, a.n, lane, mq, zq);
+        if (!(zp > 0.0) || !(zp < (double)INFINITY) || !(mp == mp)) status |= warp_row_stats(drow, a.n, lane, mp, zp);
+        if (lane == 0) accept_decide<T>(a, lr_h, pr_h, mq, zq, mp, zp, status);
+    }
+}
+
+// WPR: sweep warps that share a row (a row has up to WPR * 32 * 8 vectors of 16 bytes).  FULL: exactly that many.
+template <typename T, int WPR, bool FULL>
+__global__ void __launch_bounds__((kACW + kAFin + 1) * 32, 1) verify_accept_kernel(const __grid_constant__ VerifyArgs a)
 {
     typedef Vec<T> V;
     constexpr int VEC = Elem<T>::kVec;
     constexpr int NPV = V::kPairs;
-    constexpr int kStageBytes = kVThreads * JV * 16;
+    constexpr int GROUPS = kACW / WPR;
+    constexpr int ROWL = WPR * 32;
+    constexpr int SB = ROWL * kAJV * 16;
+    constexpr int S = accept_stages(SB);
+    typedef AControl<S, WPR> Ctl;
+    static_assert(S >= 3 && (size_t)S * SB + sizeof(Ctl) <= (size_t)kASmem, "the ring and its slots must fit in shared memory");
     extern __shared__ __align__(128) unsigned char smem[];
-    VShared &sh = *reinterpret_cast<VShared *>(smem + (size_t)kVStages * kStageBytes);
+    Ctl &sh = *reinterpret_cast<Ctl *>(smem + (size_t)S * SB);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int total = a.ws.tested[a.rows];  // written by the plan kernel
+    const int stride = gridDim.x;
+    const int nk = blockIdx.x < total ? (total - 1 - (int)blockIdx.x) / stride + 1 : 0;  // rows this CTA walks
+    const long long limit = kWaitCycles;
+
     if (tid == 0) {
-#pragma unroll
-        for (int s = 0; s < kVStages; ++s) mbar_init(&sh.full[s], 1);
+        for (int s = 0; s < S; ++s) {
+            mbar_init(&sh.slot[s].full, 1);
+            mbar_init(&sh.slot[s].swept, WPR);
+            mbar_init(&sh.slot[s].empty, 1);
+        }
         sh.abort = 0;
+        sh.issued = 0;
+        for (int f = 0; f < kAFin; ++f) sh.fin_next[f] = f;
         mbar_init_fence();
     }
     __syncthreads();
-    const int nvec = a.n / VEC;
-    const uint32_t row_bytes = (uint32_t)nvec * 16u;
-    int nj = JV;
-    if (!FULL) {
-        nj = (nvec - tid + kVThreads - 1) / kVThreads;
-        nj = nj < 0 ? 0 : (nj > JV ? JV : nj);
-    }
-    const T *tbase = reinterpret_cast<const T *>(a.target) + a.vb;
-    const int total = a.ws.tested[a.rows];  // written by the plan kernel
-    const int stride = gridDim.x;
 
-    auto issue = [&](int k) {  // thread 0: copy this CTA's k-th tested row into its stage
-        const int idx = blockIdx.x + k * stride;
-        if (idx < total) {
-            int64_t pr;
-            map_row(a.rm, a.ws.tested[idx], pr);
-            const int s = k % kVStages;
-            mbar_arrive_expect_tx(&sh.full[s], row_bytes);
-            bulk_copy_g2s(smem + (size_t)s * kStageBytes, tbase + pr * a.row_stride, row_bytes, &sh.full[s]);
+    if (warp > kAFin) {
+        // ---- a sweep warp: the maximum of its share, then the sum of exponentials about it
+        const int cw = warp - kAFin - 1, g = cw / WPR, w = cw % WPR;
+        const int v0 = w * 32 + lane;
+        int nj = kAJV;
+        if (!FULL) {
+            nj = (a.n / VEC - v0 + ROWL - 1) / ROWL;
+            nj = nj < 0 ? 0 : (nj > kAJV ? kAJV : nj);
         }
-    };
-    auto finish_parked = [&](int count) {
-        __syncthreads();
-        if (warp < count) accept_row<T>(a, sh.park[warp], lane);
-        __syncthreads();
-    };
-    if (tid == 0) {
+        for (int k = g; k < nk; k += GROUPS) {
+            const int s = k % S;
+            ASlot<WPR> &sl = sh.slot[s];
+            const unsigned char *stage = smem + (size_t)s * SB;
+            if (!wait_phase(&sl.full, (uint32_t)(k / S) & 1u, &sh.abort, limit)) break;
+            typename V::Max mx = V::max_init();
 #pragma unroll
-        for (int s = 0; s < kVStages; ++s) issue(s);
-    }
-    uint32_t phases = 0;
-    int k = 0, filled = 0;
-    bool aborted = false;
-    // Waits for this CTA's kk-th row to land and takes the maximum over it (sweep 1): each warp's maximum goes
-    // to the slot of the row's parity.  Thread 0 also clears the row's count of maxima.  Returns the thread's maximum.
-    auto first_sweep = [&](int kk) -> float {
-        const int s = kk % kVStages;
-        const unsigned char *stage = smem + (size_t)s * kStageBytes;
-        if (mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kWaitCycles)) phases ^= 1u << s;
-        else sh.abort = 1;
-        typename V::Max mx = V::max_init();
+            for (int j = 0; j < kAJV; ++j)
+                if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, v0 + j * ROWL));
+            const float mw = warp_redux_max(V::max_value(mx));
+            float2 z2 = f2(0.f);
+            if (mw > -INFINITY && mw < INFINITY) {
+                const float2 L2 = f2(kLog2e), nm2 = f2(-(mw * kLog2e));
 #pragma unroll
-        for (int j = 0; j < JV; ++j)
-            if (FULL || j < nj) mx = V::fold_max(mx, stage_vec(stage, tid + j * kVThreads));
-        const float tmax = V::max_value(mx);
-        const float wm = warp_redux_max(tmax);
-        if (lane == 0) sh.wmax[kk & 1][warp] = wm;
-        if (tid == 0) sh.nmax[kk & 3] = 0;
-        return tmax;
-    };
-    const int mine = blockIdx.x < total ? (total - 1 - (int)blockIdx.x) / stride + 1 : 0;  // rows this CTA walks
-    float tm = 0.f;  // this thread's maximum of the row being summed
-    if (mine > 0) {
-        tm = first_sweep(0);
-        __syncwarp();
-        __syncthreads();
-        if (sh.abort) aborted = true;
-    }
-    // One barrier per row: the maximum sweep of the row after this one runs before it, so the barrier that
-    // completes this row's sum also publishes the next row's maximum.
-    for (; k < mine && !aborted; ++k) {
-        const int s = k % kVStages;
-        const int par = k & 1;
-        const unsigned char *stage = smem + (size_t)s * kStageBytes;
-        const float m = warp_redux_max(sh.wmax[par][lane & (kVWarps - 1)]);
-        float tmn = 0.f;
-        if (k + 1 < mine) tmn = first_sweep(k + 1);
-        // sweep 2: sum of exponentials; terms equal to the maximum's are counted, not summed
-        const float m2 = m * kLog2e;
-        const float e0 = ex2_approx(fmaf(m, kLog2e, -m2));
-        float2 z2 = f2(0.f);
-        {
-            const float2 L2 = f2(kLog2e), nm2 = f2(-m2);
+                for (int j = 0; j < kAJV; ++j) {
+                    if (FULL || j < nj) {
+                        float2 c[NPV];
+                        V::pairs(stage_vec(stage, v0 + j * ROWL), c);
 #pragma unroll
-            for (int j = 0; j < JV; ++j) {
-                if (FULL || j < nj) {
-                    float2 c[NPV];
-                    V::pairs(stage_vec(stage, tid + j * kVThreads), c);
-#pragma unroll
-                    for (int q = 0; q < NPV; ++q) {
-                        const float2 d = __ffma2_rn(c[q], L2, nm2);
-                        z2 = __fadd2_rn(z2, make_float2(ex2_approx(d.x), ex2_approx(d.y)));
+                        for (int q = 0; q < NPV; ++q) {
+                            const float2 d = __ffma2_rn(c[q], L2, nm2);
+                            z2 = __fadd2_rn(z2, make_float2(ex2_approx(d.x), ex2_approx(d.y)));  // a NaN logit poisons the sum on purpose
+                        }
                     }
                 }
             }
-        }
-        float zs = z2.x + z2.y;
-        // A thread holding a maximum has its sum formed again without the maxima (kept exactly, as a count): a term
-        // near 1 would cost the small terms their low bits.  The whole warp does it for the thread, a code per lane.
-        for (unsigned holders = __ballot_sync(0xffffffffu, tm == m); holders != 0; holders &= holders - 1) {
-            const int h = __ffs((int)holders) - 1;
-            const int htid = (tid & ~31) + h;
-            const int hn = (FULL ? JV : __shfl_sync(0xffffffffu, nj, h)) * VEC;  // the thread's codes
-            float zz = 0.f;
-            int cnt = 0;
-            for (int i = lane; i < hn; i += 32) {
-                const T *v = reinterpret_cast<const T *>(stage + (size_t)(htid + (i / VEC) * kVThreads) * 16);
-                const float ev = ex2_approx(fmaf(Elem<T>::widen(v[i % VEC]), kLog2e, -m2));
-                if (ev == e0) ++cnt; else zz += ev;
+            const float wz = warp_sum_f(z2.x + z2.y);
+            if (lane == 0) {
+                sl.wmax[w] = mw;
+                sl.wz[w] = wz;
+                mbar_arrive(&sl.swept);
             }
-            zz = warp_sum_f(zz);
-            cnt = __reduce_add_sync(0xffffffffu, cnt);
-            if (lane == h) zs = zz;
-            if (lane == 0 && cnt > 0) atomicAdd(&sh.nmax[k & 3], cnt);
         }
-        const float wz = warp_sum_f(zs);
-        VParked &pk = sh.park[filled];
-        if (lane == 0) pk.wz[warp] = wz;
-        __syncthreads();  // every thread has read the stage, the count of maxima is complete, the next maximum is out
-        if (sh.abort) {
-            aborted = true;
-            break;
+    } else if (warp < kAFin) {
+        // ---- a finishing warp: joins the warps' sums, hands the stage back, files the row; accept tests by the batch
+        ABatch &bt = sh.batch[warp];
+        int filled = 0, k = warp;
+        for (; k < nk; k += kAFin) {
+            const int s = k % S;
+            ASlot<WPR> &sl = sh.slot[s];
+            if (!wait_phase(&sl.swept, (uint32_t)(k / S) & 1u, &sh.abort, limit)) break;
+            const float wm = sl.wmax[lane % WPR];
+            const float m = warp_redux_max(wm);
+            // a share without a finite code adds nothing; a +inf or NaN anywhere makes the sum unusable, as it must be
+            float x = 0.f;
+            if (lane < WPR && wm > -INFINITY) x = ex2_approx(wm * kLog2e - m * kLog2e) * sl.wz[lane];
+#pragma unroll
+            for (int o = WPR / 2; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            if (lane == 0) {
+                bt.lr[filled] = sl.lr;
+                bt.m[filled] = m;
+                bt.z[filled] = x;
+                mbar_arrive(&sl.empty);
+            }
+            if (++filled == kABatch) {
+                __syncwarp();
+                accept_batch<T>(a, bt, filled, lane);
+                __syncwarp();
+                filled = 0;
+            }
         }
-        if (tid == 0) {
+        __syncwarp();
+        if (filled > 0) accept_batch<T>(a, bt, filled, lane);
+        if (lane == 0) sh.fin_next[warp] = k;
+    } else if (lane == 0) {
+        // ---- the producer
+        const uint32_t row_bytes = (uint32_t)(a.n / VEC) * 16u;
+        const T *tbase = reinterpret_cast<const T *>(a.target) + a.vb;
+        int64_t lr_n = nk > 0 ? a.ws.tested[blockIdx.x] : -1, pr_n = 0;
+        if (nk > 0) map_row(a.rm, lr_n, pr_n);
+        for (int k = 0; k < nk; ++k) {
+            const int s = k % S;
+            ASlot<WPR> &sl = sh.slot[s];
+            const int64_t lr = lr_n, pr = pr_n;
+            if (k + 1 < nk) {  // the next row's place, fetched early
+                lr_n = a.ws.tested[blockIdx.x + (k + 1) * stride];
+                map_row(a.rm, lr_n, pr_n);
+            }
+            if (k >= S && !wait_phase(&sl.empty, (uint32_t)(k / S - 1) & 1u, &sh.abort, limit)) break;
+            sl.lr = lr;
             fence_proxy_async_smem();
-            issue(k + kVStages);
-            pk.lr = a.ws.tested[blockIdx.x + k * stride];
-            pk.m = m;
-            pk.e0 = e0;
-            pk.nmax = sh.nmax[k & 3];
+            mbar_arrive_expect_tx(&sl.full, row_bytes);
+            bulk_copy_g2s(smem + (size_t)s * SB, tbase + pr * a.row_stride, row_bytes, &sl.full);
+            sh.issued = k + 1;
         }
-        if (++filled == kVPark) {
-            finish_parked(filled);
-            filled = 0;
-        }
-        tm = tmn;
     }
-    if (filled > 0) finish_parked(filled);
-    if (aborted && tid == 0) {
-        // A copy never arrived: the rows this CTA still owed are marked, and the copies in flight
-        // get a last bounded chance to land before the CTA leaves.
+    __syncthreads();
+
+    if (sh.abort && tid == 0) {
+        // A copy never arrived: the rows this CTA still owed are marked, and the copies in flight get a last bounded
+        // chance to land before the CTA leaves.
         uint8_t *accept_arr = a.out.accept ? a.out.accept : a.ws.accept;
-        for (int k2 = k;; ++k2) {
-            const int idx = blockIdx.x + k2 * stride;
-            if (idx >= total) break;
-            const int64_t lr = a.ws.tested[idx];
+        int kmin = nk;
+        for (int f = 0; f < kAFin; ++f) kmin = min(kmin, sh.fin_next[f]);
+        for (int k = kmin; k < nk; ++k) {
+            const int64_t lr = a.ws.tested[blockIdx.x + k * stride];
             accept_arr[lr] = 0;
             a.ws.tq_sum[lr] = __int_as_float(0x7fc00000);
             if (a.out.row_status) a.out.row_status[lr] = CIAR_ROW_TIMEOUT;
         }
-        for (int s = 0; s < kVStages; ++s) mbar_wait_bounded(&sh.full[s], (phases >> s) & 1u, kDrainCycles);
+        const int issued = sh.issued;
+        for (int k = max(0, issued - S); k < issued; ++k)
+            mbar_wait_bounded(&sh.slot[k % S].full, (uint32_t)(k / S) & 1u, kDrainCycles);
     }
 }
 
@@ -555,27 +626,38 @@ __global__ void __launch_bounds__(kWinThreads) verify_window_kernel(VerifyArgs a
     }
 }
 
-template <typename T, int JV>
-cudaError_t launch_accept(const VerifyArgs &a, cudaStream_t stream, bool full)
+template <typename T, int WPR, bool FULL>
+cudaError_t launch_accept_one(const VerifyArgs &a, cudaStream_t stream)
 {
-    constexpr size_t smem = (size_t)kVStages * kVThreads * JV * 16 + sizeof(VShared);
-    static bool configured[64][2] = {};
+    constexpr int SB = WPR * 32 * kAJV * 16;
+    constexpr int S = accept_stages(SB);
+    constexpr size_t smem = (size_t)S * SB + sizeof(AControl<S, WPR>);
+    static bool configured[64] = {};
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!configured[dev][full]) {
-        err = full ? cudaFuncSetAttribute(verify_accept_kernel<T, JV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                   : cudaFuncSetAttribute(verify_accept_kernel<T, JV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (!configured[dev]) {
+        err = cudaFuncSetAttribute(verify_accept_kernel<T, WPR, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
-        configured[dev][full] = true;
+        configured[dev] = true;
     }
-    const int64_t cap = (int64_t)sm_count() * 2;
+    const int64_t cap = sm_count();
     const unsigned grid = (unsigned)(a.rows < cap ? a.rows : cap);
-    if (full) verify_accept_kernel<T, JV, true><<<grid, kVThreads, smem, stream>>>(a);
-    else verify_accept_kernel<T, JV, false><<<grid, kVThreads, smem, stream>>>(a);
+    verify_accept_kernel<T, WPR, FULL><<<grid, (kACW + kAFin + 1) * 32, smem, stream>>>(a);
     count_launch();
     return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_accept(const VerifyArgs &a, cudaStream_t stream)
+{
+    const int nvec = a.n / Elem<T>::kVec;
+    const int per_warp = 32 * kAJV;  // vectors one warp takes
+    if (nvec <= 2 * per_warp) return nvec == 2 * per_warp ? launch_accept_one<T, 2, true>(a, stream) : launch_accept_one<T, 2, false>(a, stream);
+    if (nvec <= 4 * per_warp) return nvec == 4 * per_warp ? launch_accept_one<T, 4, true>(a, stream) : launch_accept_one<T, 4, false>(a, stream);
+    if (nvec <= 8 * per_warp) return nvec == 8 * per_warp ? launch_accept_one<T, 8, true>(a, stream) : launch_accept_one<T, 8, false>(a, stream);
+    return nvec == 16 * per_warp ? launch_accept_one<T, 16, true>(a, stream) : launch_accept_one<T, 16, false>(a, stream);
 }
 
 template <typename T>
@@ -609,16 +691,7 @@ cudaError_t launch_all(const VerifyArgs &a, cudaStream_t stream)
     count_launch();
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
-    const int nvec = a.n / Elem<T>::kVec;
-    const int jv = nvec <= kVThreads ? 1 : (nvec <= 2 * kVThreads ? 2 : (nvec <= 4 * kVThreads ? 4 : 8));
-    const bool full = nvec == kVThreads * jv;
-    if (a.n > 16384) err = launch_accept_wide<T>(a, stream);
-    else switch (jv) {
-    case 1: err = launch_accept<T, 1>(a, stream, full); break;
-    case 2: err = launch_accept<T, 2>(a, stream, full); break;
-    case 4: err = launch_accept<T, 4>(a, stream, full); break;
-    default: err = launch_accept<T, 8>(a, stream, full); break;
-    }
+    err = a.n > 16384 ? launch_accept_wide<T>(a, stream) : launch_accept<T>(a, stream);
     if (err != cudaSuccess) return err;
     const int64_t nw = a.rows / a.window;
     const int64_t cap = (int64_t)sm_count() * 4;

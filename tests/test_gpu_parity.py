@@ -709,7 +709,7 @@ def test_workload_largevocab_full_set_flags_and_stratified_sample(ciar):
     assert torch.equal(qo.flag.bool(), inp.boundary) and abs(float(qo.flag.float().mean()) - 0.30) < 0.01
     assert int(qo.row_status.sum()) == 0 and int(vo.row_status.sum()) == 0
     flag_w = qo.flag.view(-1, W)
-    first = torch.where(flag_w.any(1), flag_w.int().argmax(1), torch.full((rows // W,), W, device="cuda")).int()
+    first = torch.where(flag_w.bool().any(1), flag_w.int().argmax(1), torch.full((rows // W,), W, device="cuda")).int()
     assert torch.equal(vo.first_flag, first) and torch.equal(vo.cloud_call.bool(), first < W)
     assert bool((vo.accepted_len >= first).all()) and bool((vo.accepted_len <= W).all())
     assert torch.equal(vo.resampled_token >= 0, vo.accepted_len < W)
