@@ -81,7 +81,10 @@ __host__ __device__ constexpr int stages_for(int stage_bytes, int nfin, int wpr)
     const int batch = wpr == 2 ? (int)sizeof(RowBatch<2>) : wpr == 4 ? (int)sizeof(RowBatch<4>) : wpr == 8 ? (int)sizeof(RowBatch<8>) : (int)sizeof(RowBatch<16>);
     const int slot = wpr == 2 ? (int)sizeof(RowSlot<2>) : wpr == 4 ? (int)sizeof(RowSlot<4>) : wpr == 8 ? (int)sizeof(RowSlot<8>) : (int)sizeof(RowSlot<16>);
     int s = (kSmemBudget - 1024 - nfin * (batch + 128)) / (stage_bytes + slot);
-    return s > kMaxStages ? kMaxStages : s;
+    s = s > kMaxStages ? kMaxStages : s;
+    // a whole number of rounds of the groups: a group then meets each stage's uses in order (a warp must never wait
+    // for a phase of a barrier before it has seen the phase before it)
+    return s - s % (kCW / wpr);
 }
 
 // Sums four values over the warp with six shuffles: on return lanes 0..7 hold the sum of v0, 8..15 of v1,
@@ -884,7 +887,7 @@ __device__ __noinline__ bool collect_row(const QuantifyArgs &a, RowSlot<WPR> &sl
         int total;
         int pos = lane_prefix(__popc(mine), lane, total);
         crowded = total > 32;
-        if (!crowded) {
+        if (!crowded && total > 0) {  // (most rows have no such lane)
             for (; mine != 0; mine &= mine - 1) pairs[pos++] = lane * WPR + __ffs((int)mine) - 1;
             __syncwarp();
             // ... each is looked at by one lane: which of its kJV vectors hold such a code ...
@@ -900,7 +903,7 @@ __device__ __noinline__ bool collect_row(const QuantifyArgs &a, RowSlot<WPR> &sl
             pos = lane_prefix(__popc(vmask), lane, total);
             crowded = total > 32;
             __syncwarp();
-            if (!crowded) {
+            if (!crowded && total > 0) {
                 for (; vmask != 0; vmask &= vmask - 1) pairs[pos++] = (__ffs((int)vmask) - 1) * ROWL + sv;
                 __syncwarp();
                 // ... and each of those vectors by one lane, which notes the logits of the codes it finds
@@ -932,27 +935,35 @@ __device__ __noinline__ bool collect_row(const QuantifyArgs &a, RowSlot<WPR> &sl
         }
         // Nearly equal exponentials?  Then the central power sums, as differences of raw ones, would have lost their
         // digits: a look in float at the raw sums of the codes that enter through the series tells.
-        float a1 = 0.f, a2 = 0.f, an = 0.f;
+        float P1f = v0, P2f = v2, nuf;
+        const bool max_in_series = lane < WPR && wc > 0 && !(ew > th);
+        if (nhit == 0 && !__any_sync(0xffffffffu, max_in_series)) {
+            // (the usual case: nothing but the warps' maxima is treated exactly)
+            nuf = (float)(a.n - __reduce_add_sync(0xffffffffu, lane < WPR ? wc : 0));
+        } else {
+            float a1 = 0.f, a2 = 0.f, an = 0.f;
 #pragma unroll
-        for (int i = 0; i < kLaneHits; ++i) {
-            if (cnt > i) {
-                const float e = ex2_approx(fmaf(h[i], kLog2e, -m2));
-                a1 -= e;
-                a2 = fmaf(-e, e, a2);
-                an -= 1.f;
+            for (int i = 0; i < kLaneHits; ++i) {
+                if (cnt > i) {
+                    const float e = ex2_approx(fmaf(h[i], kLog2e, -m2));
+                    a1 -= e;
+                    a2 = fmaf(-e, e, a2);
+                    an -= 1.f;
+                }
             }
-        }
-        if (lane < WPR && wc > 0) {
-            if (ew > th) {
-                an -= (float)wc;
-            } else {
-                a1 = fmaf((float)wc, ew, a1);
-                a2 = fmaf((float)wc * ew, ew, a2);
+            if (lane < WPR && wc > 0) {
+                if (ew > th) {
+                    an -= (float)wc;
+                } else {
+                    a1 = fmaf((float)wc, ew, a1);
+                    a2 = fmaf((float)wc * ew, ew, a2);
+                }
             }
+            const float s4 = warp_sum4(a1, a2, an, 0.f, lane);
+            P1f += __shfl_sync(0xffffffffu, s4, 0);
+            P2f += __shfl_sync(0xffffffffu, s4, 8);
+            nuf = (float)a.n + __shfl_sync(0xffffffffu, s4, 16);
         }
-        const float s4 = warp_sum4(a1, a2, an, 0.f, lane);
-        const float P1f = v0 + __shfl_sync(0xffffffffu, s4, 0), P2f = v2 + __shfl_sync(0xffffffffu, s4, 8),
-                    nuf = (float)a.n + __shfl_sync(0xffffffffu, s4, 16);
         if (P1f > 0.f && !(P2f * nuf > 1.05f * P1f * P1f)) {
             central_sums<T, WPR>(stage, nvec, lane, m2, th, P1f / nuf, wc, ew, bt, col);
             status = kStatusCentral;
@@ -1009,9 +1020,12 @@ __device__ __forceinline__ void finish_rows(const QuantifyArgs &a, const unsigne
     const long long limit = a.wait_cycles;
     RowBatch<WPR> &bt = sh.batch[f];
     int filled = 0;
-    int k = f;
-    for (; k < nk; k += NFIN) {
+    int k = 0;
+    // Each stage is always served by the same finishing warp (stage s by warp s % NFIN), which takes its rows in the
+    // order of the walk: a warp then never waits for a phase of a barrier before it has seen the phase before it.
+    for (; k < nk; ++k) {
         const int s = k % S;
+        if (s % NFIN != f) continue;
         const uint32_t par = (uint32_t)(k / S) & 1u;
         RowSlot<WPR> &sl = sh.slot[s];
         if (!wait_phase(&sl.swept, par, &sh.abort, limit)) break;
@@ -1046,7 +1060,7 @@ __global__ void __launch_bounds__((kCW + NFIN + 1) * 32, 1) quantify_stream_kern
     constexpr int SB = WPR * 32 * kJV * 16;
     constexpr int S = stages_for(SB, NFIN, WPR);
     typedef Control<S, GROUPS, NFIN, WPR> Ctl;
-    static_assert(S >= 3 && (size_t)S * SB + sizeof(Ctl) <= (size_t)kSmemBudget, "the ring and its slots must fit in shared memory");
+    static_assert(S >= 3 && S % GROUPS == 0 && (size_t)S * SB + sizeof(Ctl) <= (size_t)kSmemBudget, "the ring and its slots must fit in shared memory");
     extern __shared__ __align__(128) unsigned char smem[];
     Ctl &sh = *reinterpret_cast<Ctl *>(smem + (size_t)S * SB);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;

@@ -229,10 +229,13 @@ struct AControl {
     ABatch batch[kAFin];
 };
 
-__host__ __device__ constexpr int accept_stages(int stage_bytes)
+// (a whole number of rounds of the groups, so that a group meets each stage's uses in order: a warp must never wait for
+// a phase of a barrier before it has seen the phase before it)
+__host__ __device__ constexpr int accept_stages(int stage_bytes, int groups)
 {
     int s = (kASmem - 4096) / (stage_bytes + 256);
-    return s > kAMaxStages ? kAMaxStages : s;
+    s = s > kAMaxStages ? kAMaxStages : s;
+    return s - s % groups;
 }
 
 // The accept tests of a batch, a row per lane; rows whose statistics came out unusable are then redone one by one by the
@@ -279,9 +282,9 @@ __global__ void __launch_bounds__((kACW + kAFin + 1) * 32, 1) verify_accept_kern
     constexpr int GROUPS = kACW / WPR;
     constexpr int ROWL = WPR * 32;
     constexpr int SB = ROWL * kAJV * 16;
-    constexpr int S = accept_stages(SB);
+    constexpr int S = accept_stages(SB, GROUPS);
     typedef AControl<S, WPR> Ctl;
-    static_assert(S >= 3 && (size_t)S * SB + sizeof(Ctl) <= (size_t)kASmem, "the ring and its slots must fit in shared memory");
+    static_assert(S >= 3 && S % GROUPS == 0 && (size_t)S * SB + sizeof(Ctl) <= (size_t)kASmem, "the ring and its slots must fit in shared memory");
     extern __shared__ __align__(128) unsigned char smem[];
     Ctl &sh = *reinterpret_cast<Ctl *>(smem + (size_t)S * SB);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -348,9 +351,12 @@ __global__ void __launch_bounds__((kACW + kAFin + 1) * 32, 1) verify_accept_kern
     } else if (warp < kAFin) {
         // ---- a finishing warp: joins the warps' sums, hands the stage back, files the row; accept tests by the batch
         ABatch &bt = sh.batch[warp];
-        int filled = 0, k = warp;
-        for (; k < nk; k += kAFin) {
+        // (stage s is always served by finishing warp s % kAFin, in the order of the walk: a warp never waits for a
+        // phase of a barrier before it has seen the phase before it)
+        int filled = 0, k = 0;
+        for (; k < nk; ++k) {
             const int s = k % S;
+            if (s % kAFin != warp) continue;
             ASlot<WPR> &sl = sh.slot[s];
             if (!wait_phase(&sl.swept, (uint32_t)(k / S) & 1u, &sh.abort, limit)) break;
             const float wm = sl.wmax[lane % WPR];
@@ -630,7 +636,7 @@ template <typename T, int WPR, bool FULL>
 cudaError_t launch_accept_one(const VerifyArgs &a, cudaStream_t stream)
 {
     constexpr int SB = WPR * 32 * kAJV * 16;
-    constexpr int S = accept_stages(SB);
+    constexpr int S = accept_stages(SB, kACW / WPR);
     constexpr size_t smem = (size_t)S * SB + sizeof(AControl<S, WPR>);
     static bool configured[64] = {};
     int dev = 0;
