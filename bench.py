@@ -365,7 +365,7 @@ def run_ours(args):
 NCU_TRAFFIC = {
     # captured on 2304 of the 9216 rows and scaled by the rows: profiles/quantify_percode_kernel_llamagen384.md
     ("quantify_percode_kernel", "llamagen384"): 4 * (151.1e6 + 4.7e6),
-    ("quantify_stream_kernel", "llamagen384"): 303.4e6 + 7.2e6,  # profiles/quantify_stream_kernel_llamagen384.md
+    ("quantify_stream_kernel", "llamagen384"): 302.1e6 + 4.4e6,  # profiles/quantify_stream_kernel_llamagen384.md
     # captured on 2048 of the 65536 rows and scaled by the rows (every row is handled alone): profiles/quantify_wide_kernel_largevocab.md
     ("quantify_wide_kernel", "largevocab"): 32 * (1078.5e6 + 15.1e6),
 }
