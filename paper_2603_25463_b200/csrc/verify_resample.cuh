@@ -25,9 +25,13 @@ __device__ __forceinline__ int32_t resample_row(const RowView<T> &rd, const RowV
 {
     constexpr int V = Elem<T>::kVec;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __shared__ double sh_excl;      // of the thread whose run holds the crossing: its exclusive prefix ...
+    __shared__ int32_t sh_run[2];  // ... and its run of vectors
     if (threadIdx.x == 0) {
         sh_i[0] = -1;
         sh_i[1] = 0x7fffffff;
+        sh_run[0] = sh_run[1] = 0;
+        sh_excl = 0.0;
     }
     // Thread t owns a contiguous run of vectors so that a block scan gives code-order prefixes.
     const float ratio = (float)(zq / zp);
@@ -68,38 +72,37 @@ __device__ __forceinline__ int32_t resample_row(const RowView<T> &rd, const RowV
     int32_t result;
     if (total > 0.0) {
         const double thr = (double)u_res * total;
-        // exactly one thread has excl <= thr < incl (threads with part == 0 never qualify)
+        // exactly one thread has excl <= thr < incl (threads with part == 0 never qualify): its run of vectors holds the
+        // crossing.  The first warp walks that run, a code per lane, 32 codes at a time in code order.
         if (excl <= thr && thr < incl) {
-            double cum = excl;
+            sh_run[0] = v0;
+            sh_run[1] = v1;
+            sh_excl = excl;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            const int32_t r0 = sh_run[0], ncodes = (sh_run[1] - sh_run[0]) * V;
+            double cum = sh_excl;
             int32_t pick = -1, last_pos = -1;
-            for (int32_t vi = v0; vi < v1 && pick < 0; ++vi) {
-                float tv[V], cv[V], rs[V];
-                const int32_t i0 = rt.load(vi, tv, -INFINITY);
-                rd.load(vi, cv, -INFINITY);
-                float s = 0.f;
+            for (int32_t c0 = 0; c0 < ncodes && pick < 0; c0 += 32) {
+                const int32_t e = r0 * V + c0 + lane;  // element of the row
+                float rs = 0.f;
+                if (c0 + lane < ncodes && e >= rt.vb && e < rt.vb + rt.n)
+                    rs = residual_term(Elem<T>::widen(rt.row[e]), Elem<T>::widen(rd.row[e]), mq, mp, ratio);
+                double run = (double)rs;
 #pragma unroll
-                for (int k = 0; k < V; ++k) {
-                    rs[k] = residual_term(tv[k], cv[k], mq, mp, ratio);
-                    s += rs[k];
+                for (int o = 1; o < 32; o <<= 1) {
+                    const double up = __shfl_up_sync(0xffffffffu, run, o);
+                    if (lane >= o) run += up;
                 }
-                if (cum + (double)s > thr) {
-                    double c2 = cum;
-#pragma unroll
-                    for (int k = 0; k < V; ++k) {
-                        if (rs[k] > 0.f) last_pos = i0 + k;
-                        c2 += (double)rs[k];
-                        if (pick < 0 && rs[k] > 0.f && c2 > thr) pick = i0 + k;
-                    }
-                    if (pick < 0) pick = last_pos;  // rounding: the crossing is at the vector's end
-                } else {
-                    cum += (double)s;
-#pragma unroll
-                    for (int k = 0; k < V; ++k)
-                        if (rs[k] > 0.f) last_pos = i0 + k;
-                }
+                const unsigned pos = __ballot_sync(0xffffffffu, rs > 0.f);
+                const unsigned hit = __ballot_sync(0xffffffffu, rs > 0.f && cum + run > thr);
+                if (hit) pick = r0 * V + c0 + (__ffs((int)hit) - 1) - rt.vb;
+                else if (pos) last_pos = r0 * V + c0 + (31 - __clz((int)pos)) - rt.vb;
+                cum += __shfl_sync(0xffffffffu, run, 31);
             }
-            if (pick < 0) pick = last_pos;
-            sh_i[0] = pick;
+            if (pick < 0) pick = last_pos;  // rounding: the crossing is at the run's end
+            if (lane == 0) sh_i[0] = pick;
         }
         __syncthreads();
         result = sh_i[0] >= 0 ? sh_i[0] + vb : -1;

@@ -576,6 +576,7 @@ __global__ void __launch_bounds__(kWinThreads) verify_window_kernel(VerifyArgs a
     __shared__ double scan_warp[kWinThreads / 32];
     __shared__ int sh_i[2];
     __shared__ int sh_a;
+    __shared__ float sh_f[5];  // of the first rejected row: target max / sum, draft max / sum, the uniform of its resampling
     const T *dbase = reinterpret_cast<const T *>(a.draft);
     const T *tbase = reinterpret_cast<const T *>(a.target);
     const uint8_t *accept_arr = a.out.accept ? a.out.accept : a.ws.accept;
@@ -583,23 +584,46 @@ __global__ void __launch_bounds__(kWinThreads) verify_window_kernel(VerifyArgs a
     for (int64_t w = blockIdx.x; w < nw; w += gridDim.x) {
         const int32_t wlen = window_len(a.rm, w);
         const int64_t row0 = w * a.window;
-        if (threadIdx.x < 32) {  // the first warp scans the window, a row per lane: the loads go out together
+        if (threadIdx.x < 32) {
+            // The first warp scans the window, a row per lane.  Every load a lane may need goes out at once: its row's flag
+            // and accept bit, and the statistics and the uniform the resampling would use if this row is the first rejected.
             const int lane = threadIdx.x;
-            int32_t f = 0;
-            if (a.mode != CIAR_VERIFY_ALL) {
-                f = wlen;
-                for (int32_t base = 0; base < wlen && f == wlen; base += 32) {
-                    const int32_t j = base + lane;
-                    const unsigned mk = __ballot_sync(0xffffffffu, j < wlen && a.flag[row0 + j] != 0);
+            int32_t f = 0, acc_len = wlen;
+            if (a.mode != CIAR_VERIFY_ALL) f = wlen;
+            for (int32_t base = 0; base < wlen; base += 32) {
+                const int32_t j = base + lane;
+                const bool in = j < wlen;
+                const int64_t lr = row0 + j;
+                const uint8_t fl = in && a.flag ? a.flag[lr] : 0, ac = in ? accept_arr[lr] : 1;
+                float s_mq = 0.f, s_zq = 0.f, s_mp = 0.f, s_zp = 0.f, s_u = 0.f;
+                if (in) {
+                    int64_t pr;
+                    map_row(a.rm, lr, pr);
+                    s_mq = a.ws.tq_max[lr];
+                    s_zq = a.ws.tq_sum[lr];
+                    s_mp = a.draft_row_max[lr];
+                    s_zp = a.draft_sum_exp[lr];
+                    s_u = a.u_resample[pr];
+                }
+                if (a.mode != CIAR_VERIFY_ALL && f == wlen) {
+                    const unsigned mk = __ballot_sync(0xffffffffu, in && fl != 0);
                     if (mk) f = base + __ffs((int)mk) - 1;
                 }
-            }
-            int32_t acc_len = wlen;
-            for (int32_t base = 0; base < wlen && acc_len == wlen; base += 32) {
-                const int32_t j = base + lane;
-                const unsigned mk =
-                    __ballot_sync(0xffffffffu, tested_row(a.mode, j, f, wlen, a.flag, row0 + j) && accept_arr[row0 + j] == 0);
-                if (mk) acc_len = base + __ffs((int)mk) - 1;
+                bool tested = in;
+                if (a.mode == CIAR_VERIFY_ANCHORED) tested = in && j >= f;
+                else if (a.mode == CIAR_VERIFY_PER_TOKEN) tested = in && fl != 0;
+                const unsigned rej = __ballot_sync(0xffffffffu, tested && ac == 0);
+                if (rej && acc_len == wlen) {
+                    const int src = __ffs((int)rej) - 1;
+                    acc_len = base + src;
+                    if (lane == src) {
+                        sh_f[0] = s_mq;
+                        sh_f[1] = s_zq;
+                        sh_f[2] = s_mp;
+                        sh_f[3] = s_zp;
+                        sh_f[4] = s_u;
+                    }
+                }
             }
             if (lane == 0) {
                 sh_a = acc_len;
@@ -613,15 +637,13 @@ __global__ void __launch_bounds__(kWinThreads) verify_window_kernel(VerifyArgs a
             const int64_t lr = row0 + acc_len;
             int64_t pr;
             map_row(a.rm, lr, pr);
-            const float mq = a.ws.tq_max[lr];
-            const double zq = (double)a.ws.tq_sum[lr];
-            const float mp = a.draft_row_max[lr];
-            const double zp = (double)a.draft_sum_exp[lr];
+            const float mq = sh_f[0], mp = sh_f[2];
+            const double zq = (double)sh_f[1], zp = (double)sh_f[3];
             // unusable logits on either side (their statistics are NaN): nothing to resample from
             if (zq > 0.0 && zq < INFINITY && zp > 0.0 && zp < INFINITY && mp == mp) {
                 const RowView<T> rd(dbase + pr * a.row_stride, a.vb, a.n);
                 const RowView<T> rt(tbase + pr * a.row_stride, a.vb, a.n);
-                tok = resample_row<T, kWinThreads>(rd, rt, mp, zp, mq, zq, a.u_resample[pr], a.vb, scan_warp, sh_i);
+                tok = resample_row<T, kWinThreads>(rd, rt, mp, zp, mq, zq, sh_f[4], a.vb, scan_warp, sh_i);
             }
         }
         if (threadIdx.x == 0) {
