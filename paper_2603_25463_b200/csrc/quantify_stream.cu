@@ -1169,7 +1169,7 @@ cudaError_t launch_typed(const QuantifyArgs &a, cudaStream_t stream)
     const int nvec = a.n / Elem<T>::kVec;
     const int per_warp = 32 * kJV;  // vectors one warp takes
     if (nvec <= 2 * per_warp) return nvec == 2 * per_warp ? launch_one<T, 2, 3, true>(a, stream) : launch_one<T, 2, 3, false>(a, stream);
-    if (nvec <= 4 * per_warp) return nvec == 4 * per_warp ? launch_one<T, 4, 3, true>(a, stream) : launch_one<T, 4, 3, false>(a, stream);
+    if (nvec <= 4 * per_warp) return nvec == 4 * per_warp ? launch_one<T, 4, 4, true>(a, stream) : launch_one<T, 4, 4, false>(a, stream);
     if (nvec <= 8 * per_warp) return nvec == 8 * per_warp ? launch_one<T, 8, 3, true>(a, stream) : launch_one<T, 8, 3, false>(a, stream);
     return nvec == 16 * per_warp ? launch_one<T, 16, 2, true>(a, stream) : launch_one<T, 16, 2, false>(a, stream);
 }
