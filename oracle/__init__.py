@@ -24,6 +24,7 @@ RADIUS_SCALAR, RADIUS_PER_ROW, RADIUS_PER_CODE = 0, 1, 2
 POLICY_INTERVAL, POLICY_ENTROPY, POLICY_MAXPROB, POLICY_RANDOM, POLICY_ALL = 0, 1, 2, 3, 4
 VERIFY_ANCHORED, VERIFY_PER_TOKEN, VERIFY_ALL = 0, 1, 2
 ROW_NAN, ROW_NO_FINITE, ROW_BAD_TOKEN = 1, 2, 4
+SCORE_PRODUCT, SCORE_PER_N, SCORE_PER_OMEGA2, SCORE_SMOOTHED, SCORE_ADDITIVE = 0, 1, 2, 3, 4
 
 _lib = None
 
@@ -49,6 +50,8 @@ def lib() -> ctypes.CDLL:
         _lib.orc_verify.restype = ctypes.c_int
         _lib.orc_decode_step.restype = ctypes.c_int
         _lib.orc_max_threads.restype = ctypes.c_int
+        for name in ("orc_topk", "orc_score_variant", "orc_ensemble", "orc_vote", "orc_interdro"):
+            getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
 
@@ -264,3 +267,146 @@ def decode_step(state: DecodeState, draft_pool, target_pool, draft_token_pool, u
         ctypes.c_int(threads))
     if rc != 0:
         raise ValueError("orc_decode_step: invalid arguments (code %d)" % rc)
+
+
+@dataclass
+class TopkResult:
+    kth_logit: np.ndarray
+    n_above: np.ndarray
+    mass: np.ndarray
+    entropy: np.ndarray
+    S_lo: np.ndarray
+    S_up: np.ndarray
+    omega: np.ndarray
+    sigma: np.ndarray
+    score: np.ndarray
+    flag: np.ndarray
+    row_status: np.ndarray
+    margin: np.ndarray
+    indices: Optional[np.ndarray] = None
+
+
+def topk(logits, k: int, params: IntervalParams, valid_begin: int = 0, valid_count: Optional[int] = None,
+         indices: bool = False, threads: int = 0) -> TopkResult:
+    """Discrete top-k quantifier: full sort of every row, the interval score of the k kept codes."""
+    c, code = as_host(logits)
+    rows, vocab = c.shape
+    n = vocab - valid_begin if valid_count is None else valid_count
+    rad = _radius_host(params, code)
+    d = lambda: np.empty(rows, dtype=np.float64)
+    out = TopkResult(d(), np.empty(rows, np.int32), d(), d(), d(), d(), d(), d(), d(),
+                     np.empty(rows, np.uint8), np.empty(rows, np.uint8), d())
+    if indices:
+        out.indices = np.empty((rows, k), np.int32)
+    rc = lib().orc_topk(
+        _ptr(c), ctypes.c_int(code), ctypes.c_int64(rows), ctypes.c_int32(vocab), ctypes.c_int64(vocab),
+        ctypes.c_int32(valid_begin), ctypes.c_int32(n), ctypes.c_int32(k),
+        ctypes.c_int(params.radius_mode), _ptr(rad), ctypes.c_int(int(params.radius_is_raw)),
+        ctypes.c_double(params.r_scalar), ctypes.c_double(params.r_max),
+        ctypes.c_double(params.lo_cap), ctypes.c_double(params.hi_cap), ctypes.c_double(params.tau),
+        _ptr(out.kth_logit), _ptr(out.n_above), _ptr(out.mass), _ptr(out.entropy),
+        _ptr(out.S_lo), _ptr(out.S_up), _ptr(out.omega), _ptr(out.sigma), _ptr(out.score),
+        _ptr(out.flag), _ptr(out.row_status), _ptr(out.margin), _ptr(out.indices), ctypes.c_int(threads))
+    if rc != 0:
+        raise ValueError("orc_topk: invalid arguments (code %d)" % rc)
+    return out
+
+
+def score_variant(omega, sigma, n: int, variant: int, eps: float = 0.0, lambda1: float = 0.0,
+                  lambda2: float = 1.0, tau: float = 0.0):
+    """Score variants of the uncertainty appendix's practical remarks; returns (value, flag, margin)."""
+    om = _plain(omega, np.float64)
+    sg = _plain(sigma, np.float64)
+    rows = om.shape[0]
+    out, flag, margin = np.empty(rows, np.float64), np.empty(rows, np.uint8), np.empty(rows, np.float64)
+    rc = lib().orc_score_variant(
+        ctypes.c_int64(rows), ctypes.c_int32(n), _ptr(om), _ptr(sg), ctypes.c_int(variant),
+        ctypes.c_double(eps), ctypes.c_double(lambda1), ctypes.c_double(lambda2), ctypes.c_double(tau),
+        _ptr(out), _ptr(flag), _ptr(margin))
+    if rc != 0:
+        raise ValueError("orc_score_variant: invalid arguments (code %d)" % rc)
+    return out, flag, margin
+
+
+@dataclass
+class EnsembleResult:
+    p_max: np.ndarray
+    entropy: np.ndarray
+    S_lo: np.ndarray
+    S_up: np.ndarray
+    omega: np.ndarray
+    sigma: np.ndarray
+    score: np.ndarray
+    flag: np.ndarray
+    row_status: np.ndarray
+    margin: np.ndarray
+    pbar: Optional[np.ndarray] = None
+
+
+def ensemble(heads, params: IntervalParams, valid_begin: int = 0, valid_count: Optional[int] = None,
+             dense: bool = False, threads: int = 0) -> EnsembleResult:
+    """Soft voting over ``heads`` ([H, rows, vocab]); ``params.radius`` is float32[H, rows] for PER_ROW."""
+    c, code = as_host(heads)
+    n_heads, rows, vocab = c.shape
+    n = vocab - valid_begin if valid_count is None else valid_count
+    rad = _plain(params.radius, np.float32) if params.radius_mode == RADIUS_PER_ROW else None
+    d = lambda: np.empty(rows, dtype=np.float64)
+    out = EnsembleResult(d(), d(), d(), d(), d(), d(), d(), np.empty(rows, np.uint8), np.empty(rows, np.uint8), d())
+    if dense:
+        out.pbar = np.empty((rows, n), np.float64)
+    rc = lib().orc_ensemble(
+        _ptr(c), ctypes.c_int(code), ctypes.c_int32(n_heads), ctypes.c_int64(rows * vocab), ctypes.c_int64(rows),
+        ctypes.c_int32(vocab), ctypes.c_int64(vocab), ctypes.c_int32(valid_begin), ctypes.c_int32(n),
+        ctypes.c_int(params.radius_mode), _ptr(rad), ctypes.c_int(int(params.radius_is_raw)),
+        ctypes.c_double(params.r_scalar), ctypes.c_double(params.r_max),
+        ctypes.c_double(params.lo_cap), ctypes.c_double(params.hi_cap), ctypes.c_double(params.tau),
+        _ptr(out.p_max), _ptr(out.entropy), _ptr(out.S_lo), _ptr(out.S_up),
+        _ptr(out.omega), _ptr(out.sigma), _ptr(out.score), _ptr(out.flag), _ptr(out.row_status),
+        _ptr(out.margin), _ptr(out.pbar), ctypes.c_int(threads))
+    if rc != 0:
+        raise ValueError("orc_ensemble: invalid arguments (code %d)" % rc)
+    return out
+
+
+def vote(flags):
+    """Hard voting: flags uint8[H, rows] -> (flag uint8[rows], votes int32[rows])."""
+    f = _plain(flags, np.uint8)
+    n_heads, rows = f.shape
+    out, votes = np.empty(rows, np.uint8), np.empty(rows, np.int32)
+    rc = lib().orc_vote(ctypes.c_int32(n_heads), ctypes.c_int64(rows), _ptr(f), _ptr(out), _ptr(votes))
+    if rc != 0:
+        raise ValueError("orc_vote: invalid arguments (code %d)" % rc)
+    return out, votes
+
+
+@dataclass
+class InterDroResult:
+    l1: np.ndarray       # [3, rows]: mid, up, lo
+    ce: np.ndarray       # [3, rows]
+    kl: np.ndarray       # [rows]
+    weights: np.ndarray  # [rows]
+    loss: np.ndarray     # total, centre, upper, lower, dro, align
+
+
+def interdro(center, radius, cloud, radius_is_raw: bool = True, r_max: float = 10.0, lambda_v: float = 1.0,
+             lambda_p: float = 1.0, lambda_beta: float = 1.0, alpha: float = 1.0, valid_begin: int = 0,
+             valid_count: Optional[int] = None, threads: int = 0) -> InterDroResult:
+    """Forward value of the Inter-DRO loss over a batch of rows (one radius per code)."""
+    c, code = as_host(center)
+    r, code_r = as_host(radius)
+    t, code_t = as_host(cloud)
+    if not (code == code_r == code_t) or not (c.shape == r.shape == t.shape):
+        raise TypeError("centre, radius and cloud logits must share dtype and shape")
+    rows, vocab = c.shape
+    n = vocab - valid_begin if valid_count is None else valid_count
+    out = InterDroResult(np.empty((3, rows), np.float64), np.empty((3, rows), np.float64),
+                         np.empty(rows, np.float64), np.empty(rows, np.float64), np.empty(6, np.float64))
+    rc = lib().orc_interdro(
+        _ptr(c), _ptr(r), _ptr(t), ctypes.c_int(code), ctypes.c_int64(rows), ctypes.c_int32(vocab),
+        ctypes.c_int64(vocab), ctypes.c_int32(valid_begin), ctypes.c_int32(n),
+        ctypes.c_int(int(radius_is_raw)), ctypes.c_double(r_max),
+        ctypes.c_double(lambda_v), ctypes.c_double(lambda_p), ctypes.c_double(lambda_beta), ctypes.c_double(alpha),
+        _ptr(out.l1), _ptr(out.ce), _ptr(out.kl), _ptr(out.weights), _ptr(out.loss), ctypes.c_int(threads))
+    if rc != 0:
+        raise ValueError("orc_interdro: invalid arguments (code %d)" % rc)
+    return out

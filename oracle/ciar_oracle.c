@@ -27,6 +27,15 @@
  *                  points, brute force on tiny windows.
  *   orc_decode_step pinned: replay against orc_verify window by window and the
  *                  conservation law (every request emits exactly seq_len tokens).
+ *   orc_topk       (discrete top-k quantifier) pinned: brute-force rank counting on
+ *                  V <= 64, k = V reproducing orc_quantify, k = 1, closed forms on constant
+ *                  and geometric rows.  That it is the discrete method the paper timed:
+ *                  parity unpinned (the paper prints no formula for it).
+ *   orc_score_variant pinned: the appendix's scaling claim, the reductions to the product.
+ *   orc_ensemble / orc_vote pinned: one head and identical heads reproducing
+ *                  orc_quantify, a two-head example with a uniform average, head order.
+ *   orc_interdro   pinned: library log-softmax / relative entropy, CE = H + KL, V = 2
+ *                  closed forms, constant radius, alpha = 0 and large alpha.
  *   The operating point tau = 0.30 and the paper's end-to-end ratios depend on
  *   trained weights and data: parity unpinned (context only).
  */
@@ -619,4 +628,426 @@ int orc_max_threads(void)
 #else
     return 1;
 #endif
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Discrete top-k quantifier (the "Discrete" rows of the paper's discrete-vs-continuous
+ * comparison, k = 100 .. 400).  The paper gives no formula for it; the reading taken here:
+ * the solution set of a row is T_k = its k most probable codes (largest logits, equal
+ * logits by lowest index), found by a FULL SORT of the row; the row's discrete uncertainty
+ * is the interval score of the quantifier above applied to the k kept codes alone
+ * (softmax renormalised over T_k, n = k).  Also reported: the k-th largest logit, how many
+ * codes lie strictly above it, the mass of T_k under the full-row softmax, and the
+ * Shannon entropy of the renormalised distribution.
+ *
+ * Parity status: pinned by brute-force rank counting on V <= 64, k = V (must reproduce
+ * orc_quantify), k = 1 (mass = p_max, Omega = 0.02, U = 0), closed forms for constant and
+ * geometric rows.  That this is the discrete method the paper timed: parity unpinned.
+ * ---------------------------------------------------------------------------------------- */
+typedef struct {
+    double v;
+    int32_t i;
+} orc_kv;
+
+static int cmp_value_desc_index_asc(const void *a, const void *b)
+{
+    const orc_kv *x = (const orc_kv *)a, *y = (const orc_kv *)b;
+    if (x->v > y->v) return -1;
+    if (x->v < y->v) return 1;
+    return (x->i > y->i) - (x->i < y->i);
+}
+
+static int cmp_int32_asc(const void *a, const void *b)
+{
+    int32_t x = *(const int32_t *)a, y = *(const int32_t *)b;
+    return (x > y) - (x < y);
+}
+
+int orc_topk(const void *logits, int dtype, int64_t rows, int32_t vocab, int64_t row_stride,
+             int32_t valid_begin, int32_t valid_count, int32_t k,
+             int radius_mode, const void *radius, int radius_is_raw, double r_scalar,
+             double r_max, double lo_cap, double hi_cap, double tau,
+             double *kth_logit, int32_t *n_above, double *mass, double *entropy,
+             double *S_lo, double *S_up, double *omega, double *sigma, double *score,
+             uint8_t *flag, uint8_t *row_status, double *margin,
+             int32_t *indices /* [rows, k] ascending global code ids, nullable */, int threads)
+{
+    if (rows < 0 || valid_count < 1 || valid_begin < 0 || valid_begin + (int64_t)valid_count > vocab)
+        return 1;
+    if (k < 1 || k > valid_count) return 1;
+    orc_tensor t = { logits, dtype, rows, vocab, row_stride, valid_begin, valid_count };
+    const int32_t n = valid_count;
+#ifdef _OPENMP
+    if (threads > 0) omp_set_num_threads(threads);
+#endif
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *buf = (double *)malloc(sizeof(double) * ((size_t)n * 2 + (size_t)k * 5));
+        orc_kv *kv = (orc_kv *)malloc(sizeof(orc_kv) * (size_t)n);
+        int32_t *idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)k);
+        if (!buf || !kv || !idx) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t row = 0; row < rows; ++row) {
+            if (!buf || !kv || !idx) continue;
+            double *c = buf, *e = buf + n, *ck = buf + 2 * (size_t)n, *rk = ck + k, *ek = rk + k,
+                   *lo = ek + k, *up = lo + k;
+            int status = load_row(&t, row, c);
+            double r_row = r_scalar;
+            if (radius_mode == ORC_RADIUS_PER_ROW) r_row = (double)((const float *)radius)[row];
+            if (radius_mode != ORC_RADIUS_PER_CODE && isnan(r_row)) status |= ORC_ROW_NAN;
+            if (!status) {
+                /* full sort, most probable first */
+                for (int32_t i = 0; i < n; ++i) { kv[i].v = c[i]; kv[i].i = i; }
+                qsort(kv, (size_t)n, sizeof(orc_kv), cmp_value_desc_index_asc);
+                for (int32_t j = 0; j < k; ++j) idx[j] = kv[j].i;
+                qsort(idx, (size_t)k, sizeof(int32_t), cmp_int32_asc);
+                double kth = kv[k - 1].v;
+                int32_t above = 0;
+                for (int32_t i = 0; i < n; ++i) above += (c[i] > kth);
+                /* mass of the set under the full-row softmax */
+                double m, z;
+                softmax_row(c, n, e, &m, &z);
+                double ms = 0.0;
+                for (int32_t j = 0; j < k; ++j) ms += e[idx[j]];
+                ms /= z;
+                /* the quantifier on the kept codes alone */
+                for (int32_t j = 0; j < k; ++j) {
+                    ck[j] = c[idx[j]];
+                    if (radius_mode == ORC_RADIUS_PER_CODE) {
+                        rk[j] = load_elem(radius, dtype, row * row_stride + valid_begin + idx[j]);
+                        if (isnan(rk[j])) status |= ORC_ROW_NAN;
+                    } else {
+                        rk[j] = r_row;
+                    }
+                }
+                if (!status) {
+                    orc_row_result res;
+                    memset(&res, 0, sizeof res);
+                    quantify_row(ck, rk, k, radius_is_raw, r_max, lo_cap, hi_cap, ek, lo, up, NULL, NULL, NULL, &res);
+                    if (kth_logit) kth_logit[row] = kth;
+                    if (n_above) n_above[row] = above;
+                    if (mass) mass[row] = ms;
+                    if (entropy) entropy[row] = res.entropy;
+                    if (S_lo) S_lo[row] = res.S_lo;
+                    if (S_up) S_up[row] = res.S_up;
+                    if (omega) omega[row] = res.omega;
+                    if (sigma) sigma[row] = res.sigma;
+                    if (score) score[row] = res.score;
+                    if (flag) flag[row] = res.score > tau;
+                    if (margin) margin[row] = rel_margin(res.score, tau);
+                    if (indices)
+                        for (int32_t j = 0; j < k; ++j) indices[row * (int64_t)k + j] = idx[j] + valid_begin;
+                }
+            }
+            if (status) {
+                if (kth_logit) kth_logit[row] = NAN;
+                if (n_above) n_above[row] = -1;
+                if (mass) mass[row] = NAN;
+                if (entropy) entropy[row] = NAN;
+                if (S_lo) S_lo[row] = NAN;
+                if (S_up) S_up[row] = NAN;
+                if (omega) omega[row] = NAN;
+                if (sigma) sigma[row] = NAN;
+                if (score) score[row] = NAN;
+                if (flag) flag[row] = 1;
+                if (margin) margin[row] = INFINITY;
+                if (indices)
+                    for (int32_t j = 0; j < k; ++j) indices[row * (int64_t)k + j] = -1;
+            }
+            if (row_status) row_status[row] = (uint8_t)status;
+        }
+        free(buf);
+        free(kv);
+        free(idx);
+    }
+    return fail ? 2 : 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Score variants (uncertainty appendix, "Practical Remarks for Thresholding and
+ * Normalization"): from a row's Omega, Sigma and n,
+ *   PRODUCT     U = Omega * Sigma                       (the uncertainty-score equation)
+ *   PER_N       U / n                                    (remark 1: normalise by n)
+ *   PER_OMEGA2  U / Omega^2 = Sigma / Omega              (remark 1: normalise by Omega^2)
+ *   SMOOTHED    Omega * sqrt(Sigma^2 + eps)              (remark 2)
+ *   ADDITIVE    lambda1 * Omega + lambda2 * Omega * Sigma (remark 2)
+ * flag = variant > tau; a NaN input (unusable row) gives NaN and flag 1.
+ * Parity status: pinned by the scaling claim U(alpha delta) = alpha^2 U(delta) (PER_OMEGA2 is
+ * invariant, ADDITIVE with lambda2 = 0 is linear), eps = 0 and (lambda1, lambda2) = (0, 1)
+ * reducing to PRODUCT, and uniform widths giving Omega * sqrt(eps).
+ * ---------------------------------------------------------------------------------------- */
+#define ORC_SCORE_PRODUCT 0
+#define ORC_SCORE_PER_N 1
+#define ORC_SCORE_PER_OMEGA2 2
+#define ORC_SCORE_SMOOTHED 3
+#define ORC_SCORE_ADDITIVE 4
+
+int orc_score_variant(int64_t rows, int32_t n, const double *omega, const double *sigma, int variant,
+                      double eps, double lambda1, double lambda2, double tau,
+                      double *out, uint8_t *flag, double *margin)
+{
+    if (rows < 0 || n < 1 || variant < 0 || variant > ORC_SCORE_ADDITIVE) return 1;
+    for (int64_t row = 0; row < rows; ++row) {
+        double om = omega[row], sg = sigma[row], v;
+        switch (variant) {
+        case ORC_SCORE_PRODUCT: v = om * sg; break;
+        case ORC_SCORE_PER_N: v = om * sg / (double)n; break;
+        case ORC_SCORE_PER_OMEGA2: v = sg / om; break;
+        case ORC_SCORE_SMOOTHED: v = om * sqrt(sg * sg + eps); break;
+        default: v = lambda1 * om + lambda2 * om * sg; break;
+        }
+        if (out) out[row] = v;
+        if (flag) flag[row] = isnan(v) ? 1 : (v > tau);
+        if (margin) margin[row] = isnan(v) ? INFINITY : rel_margin(v, tau);
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Several Inter-Heads (appendix "Impact of Inter-Head Capacity").
+ * Ensemble (soft voting): the heads' probability distributions are averaged code by code,
+ *   pbar_i = (1/H) sum_h softmax(c^h)_i, and the interval is formed around the averaged
+ *   distribution (InterFuse on the logits ln pbar_i) with the mean of the heads' clamped
+ *   radii.  Reading: the paper says only that the distributions are averaged "to obtain a
+ *   calibrated score"; one radius per head and row (or one scalar) is supported.
+ * Voting (hard voting): the row is flagged when more than half of the heads flag it.
+ * heads: [H, rows, row_stride] stacked; radius: float32[H, rows] (PER_ROW) or r_scalar.
+ * Parity status: pinned by H = 1 (must reproduce orc_quantify), identical heads, a
+ * permutation of the heads, and a two-head example whose averaged distribution is uniform.
+ * ---------------------------------------------------------------------------------------- */
+int orc_ensemble(const void *heads, int dtype, int32_t n_heads, int64_t head_stride, int64_t rows,
+                 int32_t vocab, int64_t row_stride, int32_t valid_begin, int32_t valid_count,
+                 int radius_mode, const float *radius, int radius_is_raw, double r_scalar,
+                 double r_max, double lo_cap, double hi_cap, double tau,
+                 double *p_max, double *entropy, double *S_lo, double *S_up,
+                 double *omega, double *sigma, double *score, uint8_t *flag, uint8_t *row_status,
+                 double *margin, double *dense_pbar, int threads)
+{
+    if (rows < 0 || n_heads < 1 || valid_count < 1 || valid_begin < 0 || valid_begin + (int64_t)valid_count > vocab)
+        return 1;
+    if (radius_mode == ORC_RADIUS_PER_CODE) return 1;
+    const int32_t n = valid_count;
+#ifdef _OPENMP
+    if (threads > 0) omp_set_num_threads(threads);
+#endif
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *buf = (double *)malloc(sizeof(double) * (size_t)n * 7);
+        if (!buf) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t row = 0; row < rows; ++row) {
+            if (!buf) continue;
+            double *c = buf, *e = buf + n, *pbar = buf + 2 * (size_t)n, *cb = buf + 3 * (size_t)n,
+                   *rad = buf + 4 * (size_t)n, *lo = buf + 5 * (size_t)n, *up = buf + 6 * (size_t)n;
+            int status = 0;
+            double rsum = 0.0;
+            for (int32_t i = 0; i < n; ++i) pbar[i] = 0.0;
+            for (int32_t h = 0; h < n_heads; ++h) {
+                orc_tensor t = { (const char *)heads + (size_t)h * (size_t)head_stride * (dtype == ORC_F32 ? 4 : 2),
+                                 dtype, rows, vocab, row_stride, valid_begin, valid_count };
+                status |= load_row(&t, row, c);
+                double r = (radius_mode == ORC_RADIUS_PER_ROW) ? (double)radius[(int64_t)h * rows + row] : r_scalar;
+                if (isnan(r)) status |= ORC_ROW_NAN;
+                if (status) continue;
+                if (radius_is_raw) r = softplus(r);
+                if (r > r_max) r = r_max;
+                rsum += r;
+                double m, z;
+                softmax_row(c, n, e, &m, &z);
+                for (int32_t i = 0; i < n; ++i) pbar[i] += e[i] / z;
+            }
+            if (!status) {
+                for (int32_t i = 0; i < n; ++i) {
+                    pbar[i] /= (double)n_heads;
+                    cb[i] = (pbar[i] > 0.0) ? log(pbar[i]) : -INFINITY;
+                    rad[i] = rsum / (double)n_heads;
+                    if (dense_pbar) dense_pbar[row * (int64_t)n + i] = pbar[i];
+                }
+                orc_row_result res;
+                memset(&res, 0, sizeof res);
+                quantify_row(cb, rad, n, 0, r_max, lo_cap, hi_cap, e, lo, up, NULL, NULL, NULL, &res);
+                if (p_max) p_max[row] = res.p_max;
+                if (entropy) entropy[row] = res.entropy;
+                if (S_lo) S_lo[row] = res.S_lo;
+                if (S_up) S_up[row] = res.S_up;
+                if (omega) omega[row] = res.omega;
+                if (sigma) sigma[row] = res.sigma;
+                if (score) score[row] = res.score;
+                if (flag) flag[row] = res.score > tau;
+                if (margin) margin[row] = rel_margin(res.score, tau);
+            } else {
+                if (p_max) p_max[row] = NAN;
+                if (entropy) entropy[row] = NAN;
+                if (S_lo) S_lo[row] = NAN;
+                if (S_up) S_up[row] = NAN;
+                if (omega) omega[row] = NAN;
+                if (sigma) sigma[row] = NAN;
+                if (score) score[row] = NAN;
+                if (flag) flag[row] = 1;
+                if (margin) margin[row] = INFINITY;
+                if (dense_pbar)
+                    for (int32_t i = 0; i < n; ++i) dense_pbar[row * (int64_t)n + i] = NAN;
+            }
+            if (row_status) row_status[row] = (uint8_t)status;
+        }
+        free(buf);
+    }
+    return fail ? 2 : 0;
+}
+
+int orc_vote(int32_t n_heads, int64_t rows, const uint8_t *flags /* [H, rows] */, uint8_t *out, int32_t *votes)
+{
+    if (n_heads < 1 || rows < 0) return 1;
+    for (int64_t row = 0; row < rows; ++row) {
+        int32_t cnt = 0;
+        for (int32_t h = 0; h < n_heads; ++h) cnt += flags[(int64_t)h * rows + row] != 0;
+        if (votes) votes[row] = cnt;
+        if (out) out[row] = (uint8_t)(2 * cnt > n_heads);
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Inter-DRO loss, forward value (method section, paragraph "Inter-DRO Loss").
+ * Per sample (row) n, with centre logits c, radius r = min(Softplus(rho), r_max) per code,
+ * cloud logits t:   o_mid = c, o_up = c + r, o_lo = c - r   (Inter-Head: the logit interval),
+ *   p_x = softmax(o_x) for x in {mid, up, lo},  p_cloud = softmax(t),
+ *   L1_x  = sum_i |p_x,i - p_cloud,i|,
+ *   CE_x  = - sum_i p_cloud,i ln p_x,i          (terms with p_cloud,i = 0 are 0),
+ *   KL    = sum_i p_cloud,i (ln p_cloud,i - ln p_mid,i).
+ * Over the batch of N rows (reading: the paper writes the per-sample losses without a
+ * reduction; the mean is taken, and the DRO term is the softmax-weighted sum it prints):
+ *   anchor(x) = lambda_v mean_n L1_x + lambda_p mean_n CE_x        (anchor-loss equation)
+ *   align     = lambda_beta mean_n KL                               (alignment equation)
+ *   w_n = exp(alpha CE_lo^(n)) / sum_k exp(alpha CE_lo^(k)),  dro = sum_n w_n CE_lo^(n)
+ *   total = [anchor(mid) + align] + anchor(up) + [anchor(lo) + dro]  (complete-loss equation)
+ * l1, ce: [3, rows] in the order mid, up, lo.  loss[6] = total, centre, upper, lower, dro, align.
+ * Parity status: pinned by c = t with r = 0 (L1 = 0, KL = 0, CE = entropy of p_cloud), a
+ * constant radius (all three distributions coincide), V = 2 closed forms, CE - H = KL,
+ * alpha = 0 (dro = mean CE_lo) and large alpha (dro -> max CE_lo), library log-softmax.
+ * ---------------------------------------------------------------------------------------- */
+static double log_sum_exp(const double *o, int32_t n, double *m_out)
+{
+    double m = -INFINITY;
+    for (int32_t i = 0; i < n; ++i)
+        if (o[i] > m) m = o[i];
+    double z = 0.0;
+    for (int32_t i = 0; i < n; ++i) z += exp(o[i] - m);
+    *m_out = m;
+    return m + log(z);
+}
+
+int orc_interdro(const void *center, const void *radius, const void *cloud, int dtype, int64_t rows,
+                 int32_t vocab, int64_t row_stride, int32_t valid_begin, int32_t valid_count,
+                 int radius_is_raw, double r_max,
+                 double lambda_v, double lambda_p, double lambda_beta, double alpha,
+                 double *l1, double *ce, double *kl, double *weights, double *loss, int threads)
+{
+    if (rows < 1 || valid_count < 1 || valid_begin < 0 || valid_begin + (int64_t)valid_count > vocab)
+        return 1;
+    const int32_t n = valid_count;
+    orc_tensor tc = { center, dtype, rows, vocab, row_stride, valid_begin, valid_count };
+    orc_tensor tt = { cloud, dtype, rows, vocab, row_stride, valid_begin, valid_count };
+    double *rl1 = (double *)malloc(sizeof(double) * (size_t)rows * 3);
+    double *rce = (double *)malloc(sizeof(double) * (size_t)rows * 3);
+    double *rkl = (double *)malloc(sizeof(double) * (size_t)rows);
+    if (!rl1 || !rce || !rkl) { free(rl1); free(rce); free(rkl); return 2; }
+#ifdef _OPENMP
+    if (threads > 0) omp_set_num_threads(threads);
+#endif
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *buf = (double *)malloc(sizeof(double) * (size_t)n * 4);
+        if (!buf) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t row = 0; row < rows; ++row) {
+            if (!buf) continue;
+            double *c = buf, *t = buf + n, *r = buf + 2 * (size_t)n, *o = buf + 3 * (size_t)n;
+            load_row(&tc, row, c);
+            load_row(&tt, row, t);
+            for (int32_t i = 0; i < n; ++i) {
+                double rho = load_elem(radius, dtype, row * row_stride + valid_begin + i);
+                double rr = radius_is_raw ? softplus(rho) : rho;
+                r[i] = rr > r_max ? r_max : rr;
+            }
+            double mt;
+            double lse_t = log_sum_exp(t, n, &mt);
+            for (int x = 0; x < 3; ++x) {
+                for (int32_t i = 0; i < n; ++i) o[i] = (x == 0) ? c[i] : (x == 1) ? c[i] + r[i] : c[i] - r[i];
+                double mo;
+                double lse_o = log_sum_exp(o, n, &mo);
+                double s1 = 0.0, sce = 0.0, skl = 0.0;
+                for (int32_t i = 0; i < n; ++i) {
+                    double lp = o[i] - lse_o, lq = t[i] - lse_t; /* ln p_x,i and ln p_cloud,i */
+                    double p = exp(lp), q = exp(lq);
+                    s1 += fabs(p - q);
+                    if (q > 0.0) {
+                        sce -= q * lp;
+                        skl += q * (lq - lp);
+                    }
+                }
+                rl1[(size_t)x * rows + row] = s1;
+                rce[(size_t)x * rows + row] = sce;
+                if (x == 0) rkl[row] = skl;
+            }
+        }
+        free(buf);
+    }
+    if (!fail) {
+        double ml1[3] = { 0, 0, 0 }, mce[3] = { 0, 0, 0 }, mkl = 0.0;
+        for (int x = 0; x < 3; ++x) {
+            for (int64_t row = 0; row < rows; ++row) {
+                ml1[x] += rl1[(size_t)x * rows + row];
+                mce[x] += rce[(size_t)x * rows + row];
+            }
+            ml1[x] /= (double)rows;
+            mce[x] /= (double)rows;
+        }
+        for (int64_t row = 0; row < rows; ++row) mkl += rkl[row];
+        mkl /= (double)rows;
+        /* adversarial re-weighting of the batch by the lower bound's cross-entropy */
+        const double *cel = rce + (size_t)2 * rows;
+        double mx = -INFINITY;
+        for (int64_t row = 0; row < rows; ++row)
+            if (alpha * cel[row] > mx) mx = alpha * cel[row];
+        double zs = 0.0;
+        for (int64_t row = 0; row < rows; ++row) zs += exp(alpha * cel[row] - mx);
+        double dro = 0.0;
+        for (int64_t row = 0; row < rows; ++row) {
+            double w = exp(alpha * cel[row] - mx) / zs;
+            if (weights) weights[row] = w;
+            dro += w * cel[row];
+        }
+        double anchor_mid = lambda_v * ml1[0] + lambda_p * mce[0];
+        double anchor_up = lambda_v * ml1[1] + lambda_p * mce[1];
+        double anchor_lo = lambda_v * ml1[2] + lambda_p * mce[2];
+        double align = lambda_beta * mkl;
+        if (loss) {
+            loss[1] = anchor_mid + align;
+            loss[2] = anchor_up;
+            loss[3] = anchor_lo + dro;
+            loss[4] = dro;
+            loss[5] = align;
+            loss[0] = loss[1] + loss[2] + loss[3];
+        }
+        if (l1) memcpy(l1, rl1, sizeof(double) * (size_t)rows * 3);
+        if (ce) memcpy(ce, rce, sizeof(double) * (size_t)rows * 3);
+        if (kl) memcpy(kl, rkl, sizeof(double) * (size_t)rows);
+    }
+    free(rl1);
+    free(rce);
+    free(rkl);
+    return fail ? 2 : 0;
 }
