@@ -257,6 +257,101 @@ ciar_status ciar_decode_step(const ciar_decode_state *state, const ciar_logits_d
  */
 ciar_status ciar_test_stall(int32_t cta, int32_t row_in_walk, int64_t wait_cycles);
 
+/*
+ * Discrete top-k quantifier: the "Discrete" side of the paper's discrete-vs-continuous comparison
+ * (ablation section and its table, k = 100 .. 400).  The paper prints no formula; the reading
+ * built here: the solution set of a row is its k most probable codes (largest logits, equal logits
+ * by lowest index) and the row's discrete uncertainty is the interval score of ciar_quantify
+ * applied to those k codes alone (softmax renormalised over the set, n = k).  The set is found by
+ * a radix select over the logits' bit patterns with a shared-memory histogram, not by a sort.
+ * Outputs, each [rows], all device pointers, all nullable:
+ *   kth_logit float32: k-th largest logit; n_above int32: codes strictly above it (the set is
+ *   these plus the k - n_above lowest-index codes equal to kth_logit);
+ *   mass float32: probability of the set under the full-row softmax; entropy float32: Shannon
+ *   entropy (nats) of the renormalised distribution; S_lo, S_up, omega, sigma, score: as in
+ *   ciar_quantify_out but over the set; flag uint8 = score > tau; row_status uint8;
+ *   indices int32[rows, k]: the set's global code ids in ascending order (-1 for an unusable row).
+ * params: radius SCALAR or PER_ROW (PER_CODE: UNSUPPORTED); policy is ignored.
+ * Errors as ciar_quantify, plus INVALID_ARG for k < 1 or k > valid_count.  Needs no workspace.
+ */
+typedef struct {
+    float *kth_logit;
+    int32_t *n_above;
+    float *mass, *entropy, *S_lo, *S_up, *omega, *sigma, *score;
+    uint8_t *flag;
+    uint8_t *row_status;
+    int32_t *indices;
+} ciar_topk_out;
+
+ciar_status ciar_quantify_topk(const ciar_logits_desc *desc, const void *draft_logits, int32_t k,
+                               const ciar_interval_params *params, const ciar_topk_out *out, void *stream);
+
+/*
+ * Score variants (uncertainty appendix, "Practical Remarks for Thresholding and Normalization"),
+ * formed from the omega and sigma arrays ciar_quantify wrote (device float32[rows]):
+ *   PRODUCT Omega*Sigma; PER_N Omega*Sigma/n; PER_OMEGA2 Sigma/Omega; SMOOTHED
+ *   Omega*sqrt(Sigma^2 + eps); ADDITIVE lambda1*Omega + lambda2*Omega*Sigma.
+ * score_out float32[rows] and flag_out uint8[rows] (= value > tau; 1 for a NaN input) are nullable.
+ * Errors: INVALID_ARG (NULL omega / sigma with rows > 0, n < 1, bad variant, NaN tau).
+ */
+enum { CIAR_SCORE_PRODUCT = 0, CIAR_SCORE_PER_N = 1, CIAR_SCORE_PER_OMEGA2 = 2, CIAR_SCORE_SMOOTHED = 3, CIAR_SCORE_ADDITIVE = 4 };
+typedef struct {
+    int32_t variant;
+    float eps, lambda1, lambda2, tau;
+} ciar_score_params;
+
+ciar_status ciar_rescore(int64_t rows, int32_t n, const float *omega, const float *sigma,
+                         const ciar_score_params *params, float *score_out, uint8_t *flag_out, void *stream);
+
+/*
+ * Several Inter-Heads (appendix "Impact of Inter-Head Capacity").
+ * ciar_quantify_ensemble -- soft voting: the heads' softmax distributions are averaged code by
+ * code and the interval (InterFuse, normalisation, Omega, Sigma, U) is formed around the averaged
+ * distribution with the mean of the heads' clamped radii.  head_logits: device tensor
+ * [n_heads, rows, row_stride] (head h starts head_stride elements after head h - 1; each head
+ * follows desc).  params: radius SCALAR, or PER_ROW with radius = device float32[n_heads, rows];
+ * PER_CODE: UNSUPPORTED; policy is ignored (flag = U > tau).  1 <= n_heads <= CIAR_MAX_HEADS.
+ * Outputs taken from ciar_quantify_out: p_max (largest averaged probability), entropy (of the
+ * averaged distribution), S_lo, S_up, omega, sigma, score, flag, row_status, and dense_p (the
+ * averaged distribution, float32[rows, valid_count]); the other members must be NULL.
+ * ciar_vote -- hard voting: flags uint8[n_heads, rows] (one ciar_quantify per head wrote them);
+ * flag_out[row] = 1 when more than half of the heads flagged the row; votes_out int32[rows] nullable.
+ */
+#define CIAR_MAX_HEADS 8
+ciar_status ciar_quantify_ensemble(const ciar_logits_desc *desc, const void *head_logits, int32_t n_heads,
+                                   int64_t head_stride, const ciar_interval_params *params,
+                                   const ciar_quantify_out *out, void *stream);
+ciar_status ciar_vote(int32_t n_heads, int64_t rows, const uint8_t *flags, uint8_t *flag_out,
+                      int32_t *votes_out, void *stream);
+
+/*
+ * Forward value of the Inter-DRO loss over a batch of rows (method section, "Inter-DRO Loss": the
+ * anchor-loss, DRO re-weighting, alignment and complete-loss equations).  center, radius, cloud:
+ * device tensors that follow desc (radius = one value per code, raw rho when radius_is_raw).
+ * Per row: p_x = softmax(c), softmax(c + r), softmax(c - r) for x = mid, up, lo; p_cloud =
+ * softmax(cloud); L1_x = sum |p_x - p_cloud|; CE_x = -sum p_cloud ln p_x; KL = KL(p_cloud || p_mid).
+ * Over the batch: anchor(x) = lambda_v mean L1_x + lambda_p mean CE_x; align = lambda_beta mean KL;
+ * w = softmax(alpha CE_lo) over the rows, dro = sum w CE_lo; total = anchor(mid) + align +
+ * anchor(up) + anchor(lo) + dro.
+ * Outputs (device, nullable): l1, ce float32[3, rows] (mid, up, lo); kl, weights float32[rows];
+ * loss float32[6] = total, centre, upper, lower, dro, align.
+ * workspace: device scratch of ciar_interdro_workspace_bytes(rows) bytes, 16-byte aligned.
+ * Errors: as ciar_quantify, plus WORKSPACE_TOO_SMALL; rows must be >= 1.
+ */
+typedef struct {
+    int32_t radius_is_raw;
+    float r_max;
+    float lambda_v, lambda_p, lambda_beta, alpha;
+} ciar_interdro_params;
+typedef struct {
+    float *l1, *ce, *kl, *weights, *loss;
+} ciar_interdro_out;
+size_t ciar_interdro_workspace_bytes(int64_t rows);
+ciar_status ciar_interdro_forward(const ciar_logits_desc *desc, const void *center, const void *radius,
+                                  const void *cloud, const ciar_interdro_params *params,
+                                  const ciar_interdro_out *out, void *workspace, size_t workspace_bytes,
+                                  void *stream);
+
 /* Human-readable name of a status code (host pointer to a static string). */
 const char *ciar_status_string(ciar_status s);
 

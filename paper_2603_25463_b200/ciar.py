@@ -350,3 +350,176 @@ def decode_step(state: DecodeState, draft_pool: torch.Tensor, target_pool: torch
                                  _stream(stream))
     if st != 0:
         raise CiarError("ciar_decode_step", st)
+
+
+# ---------------------------------------------------------------- discrete top-k, score variants, several heads, Inter-DRO
+SCORE_PRODUCT, SCORE_PER_N, SCORE_PER_OMEGA2, SCORE_SMOOTHED, SCORE_ADDITIVE = 0, 1, 2, 3, 4
+MAX_HEADS = 8
+
+
+class TopkOutC(ctypes.Structure):
+    _fields_ = [(n, _vp) for n in ("kth_logit", "n_above", "mass", "entropy", "S_lo", "S_up", "omega", "sigma",
+                                   "score", "flag", "row_status", "indices")]
+
+
+class ScoreParamsC(ctypes.Structure):
+    _fields_ = [("variant", ctypes.c_int32), ("eps", ctypes.c_float), ("lambda1", ctypes.c_float),
+                ("lambda2", ctypes.c_float), ("tau", ctypes.c_float)]
+
+
+class InterDroParamsC(ctypes.Structure):
+    _fields_ = [("radius_is_raw", ctypes.c_int32), ("r_max", ctypes.c_float), ("lambda_v", ctypes.c_float),
+                ("lambda_p", ctypes.c_float), ("lambda_beta", ctypes.c_float), ("alpha", ctypes.c_float)]
+
+
+class InterDroOutC(ctypes.Structure):
+    _fields_ = [(n, _vp) for n in ("l1", "ce", "kl", "weights", "loss")]
+
+
+_extras_ready = False
+
+
+def _load_extras() -> ctypes.CDLL:
+    global _extras_ready
+    lib = load()
+    if not _extras_ready:
+        lib.ciar_quantify_topk.restype = ctypes.c_int
+        lib.ciar_quantify_topk.argtypes = [ctypes.POINTER(LogitsDesc), _vp, ctypes.c_int32,
+                                           ctypes.POINTER(IntervalParamsC), ctypes.POINTER(TopkOutC), _vp]
+        lib.ciar_rescore.restype = ctypes.c_int
+        lib.ciar_rescore.argtypes = [ctypes.c_int64, ctypes.c_int32, _vp, _vp, ctypes.POINTER(ScoreParamsC), _vp, _vp, _vp]
+        lib.ciar_quantify_ensemble.restype = ctypes.c_int
+        lib.ciar_quantify_ensemble.argtypes = [ctypes.POINTER(LogitsDesc), _vp, ctypes.c_int32, ctypes.c_int64,
+                                               ctypes.POINTER(IntervalParamsC), ctypes.POINTER(QuantifyOutC), _vp]
+        lib.ciar_vote.restype = ctypes.c_int
+        lib.ciar_vote.argtypes = [ctypes.c_int32, ctypes.c_int64, _vp, _vp, _vp, _vp]
+        lib.ciar_interdro_workspace_bytes.restype = ctypes.c_size_t
+        lib.ciar_interdro_workspace_bytes.argtypes = [ctypes.c_int64]
+        lib.ciar_interdro_forward.restype = ctypes.c_int
+        lib.ciar_interdro_forward.argtypes = [ctypes.POINTER(LogitsDesc), _vp, _vp, _vp, ctypes.POINTER(InterDroParamsC),
+                                              ctypes.POINTER(InterDroOutC), _vp, ctypes.c_size_t, _vp]
+        _extras_ready = True
+    return lib
+
+
+_T_F32 = ("kth_logit", "mass", "entropy", "S_lo", "S_up", "omega", "sigma", "score")
+
+
+@dataclass
+class TopkOut:
+    """Output tensors of ciar_quantify_topk; allocate() makes all of them."""
+    kth_logit: Optional[torch.Tensor] = None
+    n_above: Optional[torch.Tensor] = None
+    mass: Optional[torch.Tensor] = None
+    entropy: Optional[torch.Tensor] = None
+    S_lo: Optional[torch.Tensor] = None
+    S_up: Optional[torch.Tensor] = None
+    omega: Optional[torch.Tensor] = None
+    sigma: Optional[torch.Tensor] = None
+    score: Optional[torch.Tensor] = None
+    flag: Optional[torch.Tensor] = None
+    row_status: Optional[torch.Tensor] = None
+    indices: Optional[torch.Tensor] = None
+
+    @classmethod
+    def allocate(cls, rows: int, device, k: int = 0) -> "TopkOut":
+        o = cls()
+        for n in _T_F32:
+            setattr(o, n, torch.empty(rows, dtype=torch.float32, device=device))
+        o.n_above = torch.empty(rows, dtype=torch.int32, device=device)
+        o.flag = torch.empty(rows, dtype=torch.uint8, device=device)
+        o.row_status = torch.empty(rows, dtype=torch.uint8, device=device)
+        if k:
+            o.indices = torch.empty((rows, k), dtype=torch.int32, device=device)
+        return o
+
+    def to_c(self) -> TopkOutC:
+        names = [f[0] for f in TopkOutC._fields_]
+        _require_cuda(*[getattr(self, n) for n in names])
+        return TopkOutC(*[_ptr(getattr(self, n)) for n in names])
+
+
+def quantify_topk(logits: torch.Tensor, k: int, params: IntervalParams, out: TopkOut, valid_begin: int = 0,
+                  valid_count: Optional[int] = None, stream=None) -> TopkOut:
+    """ciar_quantify_topk: the discrete top-k quantifier of every row of ``logits``."""
+    _require_cuda(logits)
+    desc = make_desc(logits, valid_begin, valid_count)
+    pc, oc = params.to_c(), out.to_c()
+    st = _load_extras().ciar_quantify_topk(ctypes.byref(desc), _ptr(logits), int(k), ctypes.byref(pc), ctypes.byref(oc),
+                                           _stream(stream))
+    if st != 0:
+        raise CiarError("ciar_quantify_topk", st)
+    return out
+
+
+def rescore(omega: torch.Tensor, sigma: torch.Tensor, n: int, variant: int, eps: float = 0.0, lambda1: float = 0.0,
+            lambda2: float = 1.0, tau: float = 0.0, score_out: Optional[torch.Tensor] = None,
+            flag_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """ciar_rescore: a score variant and its flag from the omega / sigma arrays of ciar_quantify."""
+    _require_cuda(omega, sigma, score_out, flag_out)
+    pc = ScoreParamsC(int(variant), eps, lambda1, lambda2, tau)
+    st = _load_extras().ciar_rescore(omega.numel(), int(n), _ptr(omega), _ptr(sigma), ctypes.byref(pc), _ptr(score_out),
+                                     _ptr(flag_out), _stream(stream))
+    if st != 0:
+        raise CiarError("ciar_rescore", st)
+
+
+def quantify_ensemble(heads: torch.Tensor, params: IntervalParams, out: QuantifyOut, valid_begin: int = 0,
+                      valid_count: Optional[int] = None, stream=None) -> QuantifyOut:
+    """ciar_quantify_ensemble: soft voting over ``heads`` ([H, rows, vocab], contiguous)."""
+    _require_cuda(heads)
+    if heads.dim() != 3 or not heads.is_contiguous():
+        raise ValueError("heads must be a contiguous [H, rows, vocab] tensor")
+    desc = make_desc(heads[0], valid_begin, valid_count)
+    pc, oc = params.to_c(), out.to_c()
+    st = _load_extras().ciar_quantify_ensemble(ctypes.byref(desc), _ptr(heads), heads.shape[0], heads.stride(0),
+                                               ctypes.byref(pc), ctypes.byref(oc), _stream(stream))
+    if st != 0:
+        raise CiarError("ciar_quantify_ensemble", st)
+    return out
+
+
+def vote(flags: torch.Tensor, flag_out: torch.Tensor, votes_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """ciar_vote: hard voting over flags uint8[H, rows]."""
+    _require_cuda(flags, flag_out, votes_out)
+    if flags.dim() != 2 or not flags.is_contiguous() or flags.dtype != torch.uint8:
+        raise ValueError("flags must be a contiguous uint8 [H, rows] tensor")
+    st = _load_extras().ciar_vote(flags.shape[0], flags.shape[1], _ptr(flags), _ptr(flag_out), _ptr(votes_out),
+                                  _stream(stream))
+    if st != 0:
+        raise CiarError("ciar_vote", st)
+
+
+@dataclass
+class InterDroOut:
+    l1: Optional[torch.Tensor] = None       # float32[3, rows]: mid, up, lo
+    ce: Optional[torch.Tensor] = None       # float32[3, rows]
+    kl: Optional[torch.Tensor] = None       # float32[rows]
+    weights: Optional[torch.Tensor] = None  # float32[rows]
+    loss: Optional[torch.Tensor] = None     # float32[6]: total, centre, upper, lower, dro, align
+
+    @classmethod
+    def allocate(cls, rows: int, device) -> "InterDroOut":
+        f = lambda *s: torch.empty(s, dtype=torch.float32, device=device)
+        return cls(f(3, rows), f(3, rows), f(rows), f(rows), f(6))
+
+
+def interdro_workspace_bytes(rows: int) -> int:
+    return int(_load_extras().ciar_interdro_workspace_bytes(rows))
+
+
+def interdro_forward(center: torch.Tensor, radius: torch.Tensor, cloud: torch.Tensor, out: InterDroOut,
+                     workspace: torch.Tensor, radius_is_raw: bool = True, r_max: float = 10.0, lambda_v: float = 1.0,
+                     lambda_p: float = 1.0, lambda_beta: float = 1.0, alpha: float = 1.0, valid_begin: int = 0,
+                     valid_count: Optional[int] = None, stream=None) -> InterDroOut:
+    """ciar_interdro_forward: forward value of the Inter-DRO loss over the batch of rows."""
+    _require_cuda(center, radius, cloud, workspace, out.l1, out.ce, out.kl, out.weights, out.loss)
+    desc = make_desc(center, valid_begin, valid_count)
+    pc = InterDroParamsC(int(radius_is_raw), r_max, lambda_v, lambda_p, lambda_beta, alpha)
+    oc = InterDroOutC(_ptr(out.l1), _ptr(out.ce), _ptr(out.kl), _ptr(out.weights), _ptr(out.loss))
+    st = _load_extras().ciar_interdro_forward(ctypes.byref(desc), _ptr(center), _ptr(radius), _ptr(cloud), ctypes.byref(pc),
+                                              ctypes.byref(oc), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                              _stream(stream))
+    if st != 0:
+        raise CiarError("ciar_interdro_forward", st)
+    return out

@@ -337,4 +337,118 @@ ciar_status ciar_decode_step(const ciar_decode_state *state, const ciar_logits_d
     return launch_decode_update(ua, st) == cudaSuccess ? CIAR_OK : CIAR_ERR_CUDA;
 }
 
+ciar_status ciar_quantify_topk(const ciar_logits_desc *desc, const void *draft_logits, int32_t k,
+                               const ciar_interval_params *params, const ciar_topk_out *out, void *stream)
+{
+    ciar_status st = check_desc(desc, draft_logits);
+    if (st != CIAR_OK) return st;
+    st = check_interval(desc, params);
+    if (st != CIAR_OK) return st;
+    if (!out) return CIAR_ERR_INVALID_ARG;
+    if (k < 1 || k > desc->valid_count) return CIAR_ERR_INVALID_ARG;
+    if (params->radius_mode == CIAR_RADIUS_PER_CODE) return CIAR_ERR_UNSUPPORTED;
+    if (desc->rows == 0) return CIAR_OK;
+    TopkArgs a;
+    a.logits = draft_logits;
+    a.rows = desc->rows;
+    a.row_stride = desc->row_stride;
+    a.vb = desc->valid_begin;
+    a.n = desc->valid_count;
+    a.k = k;
+    a.radius_mode = params->radius_mode;
+    a.radius_is_raw = params->radius_is_raw;
+    a.radius = params->radius;
+    a.r_scalar = params->r_scalar;
+    a.r_max = params->r_max;
+    a.lo_cap = params->lo_cap;
+    a.hi_cap = params->hi_cap;
+    a.tau = params->tau;
+    a.out = *out;
+    return launch_topk(a, desc->dtype, (cudaStream_t)stream) == cudaSuccess ? CIAR_OK : CIAR_ERR_CUDA;
+}
+
+ciar_status ciar_rescore(int64_t rows, int32_t n, const float *omega, const float *sigma,
+                         const ciar_score_params *params, float *score_out, uint8_t *flag_out, void *stream)
+{
+    if (!params || rows < 0 || n < 1) return CIAR_ERR_INVALID_ARG;
+    if (params->variant < CIAR_SCORE_PRODUCT || params->variant > CIAR_SCORE_ADDITIVE) return CIAR_ERR_INVALID_ARG;
+    if (params->tau != params->tau) return CIAR_ERR_INVALID_ARG;
+    if (rows > 0 && (!omega || !sigma)) return CIAR_ERR_INVALID_ARG;
+    return launch_rescore(rows, n, omega, sigma, *params, score_out, flag_out, (cudaStream_t)stream) == cudaSuccess
+               ? CIAR_OK : CIAR_ERR_CUDA;
+}
+
+ciar_status ciar_vote(int32_t n_heads, int64_t rows, const uint8_t *flags, uint8_t *flag_out,
+                      int32_t *votes_out, void *stream)
+{
+    if (n_heads < 1 || n_heads > CIAR_MAX_HEADS || rows < 0) return CIAR_ERR_INVALID_ARG;
+    if (rows > 0 && !flags) return CIAR_ERR_INVALID_ARG;
+    return launch_vote(n_heads, rows, flags, flag_out, votes_out, (cudaStream_t)stream) == cudaSuccess
+               ? CIAR_OK : CIAR_ERR_CUDA;
+}
+
+ciar_status ciar_quantify_ensemble(const ciar_logits_desc *desc, const void *head_logits, int32_t n_heads,
+                                   int64_t head_stride, const ciar_interval_params *params,
+                                   const ciar_quantify_out *out, void *stream)
+{
+    ciar_status st = check_desc(desc, head_logits);
+    if (st != CIAR_OK) return st;
+    st = check_interval(desc, params);
+    if (st != CIAR_OK) return st;
+    if (!out) return CIAR_ERR_INVALID_ARG;
+    if (n_heads < 1 || n_heads > CIAR_MAX_HEADS) return CIAR_ERR_INVALID_ARG;
+    if (params->radius_mode == CIAR_RADIUS_PER_CODE) return CIAR_ERR_UNSUPPORTED;
+    if (n_heads > 1 && head_stride < desc->rows * desc->row_stride) return CIAR_ERR_INVALID_ARG;
+    if ((head_stride * elem_size(desc->dtype)) % 16 != 0) return CIAR_ERR_ALIGNMENT;
+    if (out->row_max || out->sum_exp || out->lse || out->argmax || out->dense_lo || out->dense_up) return CIAR_ERR_INVALID_ARG;
+    if (desc->rows == 0) return CIAR_OK;
+    EnsembleArgs a;
+    a.heads = head_logits;
+    a.n_heads = n_heads;
+    a.head_stride = head_stride;
+    a.rows = desc->rows;
+    a.row_stride = desc->row_stride;
+    a.vb = desc->valid_begin;
+    a.n = desc->valid_count;
+    a.radius_mode = params->radius_mode;
+    a.radius_is_raw = params->radius_is_raw;
+    a.radius = reinterpret_cast<const float *>(params->radius);
+    a.r_scalar = params->r_scalar;
+    a.r_max = params->r_max;
+    a.lo_cap = params->lo_cap;
+    a.hi_cap = params->hi_cap;
+    a.tau = params->tau;
+    a.out = *out;
+    return launch_ensemble(a, desc->dtype, (cudaStream_t)stream) == cudaSuccess ? CIAR_OK : CIAR_ERR_CUDA;
+}
+
+size_t ciar_interdro_workspace_bytes(int64_t rows) { return rows < 0 ? 0 : (size_t)rows * 7 * sizeof(double); }
+
+ciar_status ciar_interdro_forward(const ciar_logits_desc *desc, const void *center, const void *radius,
+                                  const void *cloud, const ciar_interdro_params *params,
+                                  const ciar_interdro_out *out, void *workspace, size_t workspace_bytes,
+                                  void *stream)
+{
+    ciar_status st = check_desc(desc, center);
+    if (st != CIAR_OK) return st;
+    if ((st = check_desc(desc, radius)) != CIAR_OK) return st;
+    if ((st = check_desc(desc, cloud)) != CIAR_OK) return st;
+    if (!params || !out || desc->rows < 1) return CIAR_ERR_INVALID_ARG;
+    if (!(params->r_max > 0.f) || !(params->r_max <= 80.f)) return CIAR_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 15u) != 0) return workspace ? CIAR_ERR_ALIGNMENT : CIAR_ERR_INVALID_ARG;
+    if (workspace_bytes < ciar_interdro_workspace_bytes(desc->rows)) return CIAR_ERR_WORKSPACE_TOO_SMALL;
+    InterDroArgs a;
+    a.center = center;
+    a.radius = radius;
+    a.cloud = cloud;
+    a.rows = desc->rows;
+    a.row_stride = desc->row_stride;
+    a.vb = desc->valid_begin;
+    a.n = desc->valid_count;
+    a.prm = *params;
+    a.out = *out;
+    a.ws = reinterpret_cast<double *>(workspace);
+    return launch_interdro(a, desc->dtype, (cudaStream_t)stream) == cudaSuccess ? CIAR_OK : CIAR_ERR_CUDA;
+}
+
 }  // extern "C"

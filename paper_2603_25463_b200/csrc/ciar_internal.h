@@ -58,7 +58,45 @@ struct DecodeUpdateArgs {
     const int32_t *first_flag, *accepted_len, *resampled_token;  // [requests]
 };
 
+struct TopkArgs {
+    const void *logits;
+    int64_t rows, row_stride;
+    int32_t vb, n, k;
+    int32_t radius_mode, radius_is_raw;
+    const void *radius;
+    float r_scalar, r_max, lo_cap, hi_cap, tau;
+    ciar_topk_out out;
+};
+
+struct EnsembleArgs {
+    const void *heads;
+    int32_t n_heads;
+    int64_t head_stride;
+    int64_t rows, row_stride;
+    int32_t vb, n;
+    int32_t radius_mode, radius_is_raw;
+    const float *radius;  // [n_heads, rows] when PER_ROW
+    float r_scalar, r_max, lo_cap, hi_cap, tau;
+    ciar_quantify_out out;
+};
+
+struct InterDroArgs {
+    const void *center, *radius, *cloud;
+    int64_t rows, row_stride;
+    int32_t vb, n;
+    ciar_interdro_params prm;
+    ciar_interdro_out out;
+    double *ws;  // [7, rows]: L1 mid / up / lo, CE mid / up / lo, KL of every row, kept in double for the batch step
+};
+
 cudaError_t launch_quantify(const QuantifyArgs &a, int dtype, cudaStream_t stream);
+cudaError_t launch_topk(const TopkArgs &a, int dtype, cudaStream_t stream);
+cudaError_t launch_rescore(int64_t rows, int32_t n, const float *omega, const float *sigma, const ciar_score_params &p,
+                           float *score_out, uint8_t *flag_out, cudaStream_t stream);
+cudaError_t launch_ensemble(const EnsembleArgs &a, int dtype, cudaStream_t stream);
+cudaError_t launch_vote(int32_t n_heads, int64_t rows, const uint8_t *flags, uint8_t *flag_out, int32_t *votes_out,
+                        cudaStream_t stream);
+cudaError_t launch_interdro(const InterDroArgs &a, int dtype, cudaStream_t stream);
 // The streaming (TMA ring) quantifier and the test that says whether it covers a call.
 bool quantify_stream_eligible(const QuantifyArgs &a, int dtype);
 cudaError_t launch_quantify_stream(const QuantifyArgs &a, int dtype, cudaStream_t stream);

@@ -2,46 +2,11 @@
 // Omega * Sigma score and the cloud flag.  One CTA per token row; the row is read from HBM once
 // (the later sweeps hit L1 / L2).
 #include "ciar_internal.h"
+#include "interval_math.cuh"
 
 namespace ciar {
 
 namespace {
-
-// Radius of a whole row as interval constants: a = exp(-r), b = exp(r), alpha = 1 - a,
-// beta = b - 1, bma = b - a (all from double so that tiny radii keep their digits).
-struct RadiusConst {
-    float a, alpha, beta, bma;
-};
-
-__device__ __forceinline__ double clamp_radius(double rho, int raw, double r_max)
-{
-    double r = rho;
-    if (raw) r = (rho > 0.0) ? rho + log1p(exp(-rho)) : log1p(exp(rho));  // Softplus, beta = 1
-    return r > r_max ? r_max : r;
-}
-
-__device__ __forceinline__ RadiusConst radius_const(double r)
-{
-    RadiusConst k;
-    const double al = -expm1(-r), be = expm1(r);
-    k.a = (float)(1.0 - al);
-    k.alpha = (float)al;
-    k.beta = (float)be;
-    k.bma = (float)(al + be);
-    return k;
-}
-
-// One code's bounds from its softmax probability p (InterFuse with the max-trick, rewritten in p):
-//   p^l = a p / (1 - alpha p),  p^u = b p / (1 + beta p),
-//   d = p^u - p^l = p (b - a)(1 - p) / ((1 - alpha p)(1 + beta p))   -- no cancellation for small r.
-__device__ __forceinline__ void bounds_from_p(float p, const RadiusConst &k, float &pl, float &d)
-{
-    const float den_l = fmaf(-k.alpha, p, 1.0f);
-    const float den_u = fmaf(k.beta, p, 1.0f);
-    const float q = __fdividef(p, den_l * den_u);
-    pl = k.a * (q * den_u);
-    d = k.bma * (q * (1.0f - p));
-}
 
 template <typename T>
 __device__ __forceinline__ RadiusConst code_radius(const RowView<T> &, float rho, int raw, float r_max)
