@@ -146,28 +146,54 @@ __global__ void __launch_bounds__(kThreads) interdro_rows_kernel(InterDroArgs a,
         const double ce_mid = lse[0] - eq_c, ce_up = lse[1] - (eq_c + eq_r), ce_lo = lse[2] - (eq_c - eq_r);
         const double kl = eq_d - (lse[3] - lse[0]);
 
-        // ---- 3. L1 distances
+        // ---- 3. L1 distances.  A code that holds more than half of the mass on both sides is left out of the
+        // sum: the difference of two probabilities near 1 has no digits left in float, while their complements
+        // (the sums over all the other codes) do, and p - q = (1 - q) - (1 - p).
         double l1[3] = { 0, 0, 0 };
+        double oth[8] = { 0, 0, 0, 0, 0, 0, 0, 0 };  // per x: sum of the other codes' p, of their q; [6] codes left out
         for (int vi = vec_begin + tid; vi < vec_end; vi += kThreads) {
             float c[V], rho[V], t[V];
             const int i0 = vc.load(vi, c, -INFINITY);
             vr.load(vi, rho, 0.f);
             vt.load(vi, t, -INFINITY);
-            float s[3] = { 0.f, 0.f, 0.f };
+            float s[3] = { 0.f, 0.f, 0.f }, sp[3] = { 0.f, 0.f, 0.f }, sq[3] = { 0.f, 0.f, 0.f };
+            int left_out = 0;
 #pragma unroll
             for (int k = 0; k < V; ++k) {
                 if (i0 + k < 0 || i0 + k >= a.n) continue;
                 const float r = code_radius_f(rho[k], raw, r_max);
                 const float q = ex2_approx(fmaf(t[k], kLog2e, -hi[3]) - lo[3]);
-                s[0] += fabsf(ex2_approx(fmaf(c[k], kLog2e, -hi[0]) - lo[0]) - q);
-                s[1] += fabsf(ex2_approx(fmaf(c[k] + r, kLog2e, -hi[1]) - lo[1]) - q);
-                s[2] += fabsf(ex2_approx(fmaf(c[k] - r, kLog2e, -hi[2]) - lo[2]) - q);
+                float px[3];
+                px[0] = ex2_approx(fmaf(c[k], kLog2e, -hi[0]) - lo[0]);
+                px[1] = ex2_approx(fmaf(c[k] + r, kLog2e, -hi[1]) - lo[1]);
+                px[2] = ex2_approx(fmaf(c[k] - r, kLog2e, -hi[2]) - lo[2]);
+#pragma unroll
+                for (int x = 0; x < 3; ++x) {
+                    if (q > 0.5f && px[x] > 0.5f) {
+                        left_out |= 1 << x;
+                    } else {
+                        s[x] += fabsf(px[x] - q);
+                        sp[x] += px[x];
+                        sq[x] += q;
+                    }
+                }
             }
-            l1[0] += (double)s[0];
-            l1[1] += (double)s[1];
-            l1[2] += (double)s[2];
+#pragma unroll
+            for (int x = 0; x < 3; ++x) {
+                l1[x] += (double)s[x];
+                oth[2 * x] += (double)sp[x];
+                oth[2 * x + 1] += (double)sq[x];
+            }
+            oth[6] += (double)left_out;  // at most one code of a row is left out per x: the bits add up without carries
         }
         block_sum<3>(l1, sh.ds);
+        block_sum<8>(oth, sh.ds);
+        {
+            const int left_out = (int)oth[6];
+#pragma unroll
+            for (int x = 0; x < 3; ++x)
+                if ((left_out >> x) & 1) l1[x] += fabs(oth[2 * x + 1] - oth[2 * x]);
+        }
         if (tid == 0) {
             const double vals[7] = { l1[0], l1[1], l1[2], ce_mid, ce_up, ce_lo, kl };
 #pragma unroll
