@@ -9,7 +9,8 @@
 //      with q_i = e_t,i / Z_t they give CE_x = lse_x - E_q[o_x] and KL = E_q[t - c] - (lse_t - lse_mid) without a
 //      pass of their own;
 //   3. the L1 distances from normalised probabilities p = 2^(o L - lse2), lse2 = m2 + log2 Z held as a float pair.
-// L is the float constant log2(e); m2 = fl(m L).
+// L is the float constant log2(e); m2 = fl(m L).  The exponent of c +- r is formed as (c L - ref) +- r L, never from
+// the float sum c + r, whose rounding (1e-6 of a logit near 30) would show in the probabilities of the large codes.
 #include "ciar_internal.h"
 
 namespace ciar {
@@ -118,8 +119,8 @@ __global__ void __launch_bounds__(kThreads) interdro_rows_kernel(InterDroArgs a,
             for (int k = 0; k < V; ++k) {
                 const float r = code_radius_f(rho[k], raw, r_max);
                 s[0] += ex2_approx(fmaf(c[k], kLog2e, -m2[0]));
-                s[1] += ex2_approx(fmaf(c[k] + r, kLog2e, -m2[1]));
-                s[2] += ex2_approx(fmaf(c[k] - r, kLog2e, -m2[2]));
+                s[1] += ex2_approx(fmaf(r, kLog2e, fmaf(c[k], kLog2e, -m2[1])));
+                s[2] += ex2_approx(fmaf(-r, kLog2e, fmaf(c[k], kLog2e, -m2[2])));
                 const float et = ex2_approx(fmaf(t[k], kLog2e, -m2[3]));
                 s[3] += et;
                 if (et > 0.f) {  // a code the cloud gives no mass: its terms are 0 whatever the device logits
@@ -165,8 +166,8 @@ __global__ void __launch_bounds__(kThreads) interdro_rows_kernel(InterDroArgs a,
                 const float q = ex2_approx(fmaf(t[k], kLog2e, -hi[3]) - lo[3]);
                 float px[3];
                 px[0] = ex2_approx(fmaf(c[k], kLog2e, -hi[0]) - lo[0]);
-                px[1] = ex2_approx(fmaf(c[k] + r, kLog2e, -hi[1]) - lo[1]);
-                px[2] = ex2_approx(fmaf(c[k] - r, kLog2e, -hi[2]) - lo[2]);
+                px[1] = ex2_approx(fmaf(r, kLog2e, fmaf(c[k], kLog2e, -hi[1])) - lo[1]);
+                px[2] = ex2_approx(fmaf(-r, kLog2e, fmaf(c[k], kLog2e, -hi[2])) - lo[2]);
 #pragma unroll
                 for (int x = 0; x < 3; ++x) {
                     if (q > 0.5f && px[x] > 0.5f) {
